@@ -1,0 +1,217 @@
+/*
+ * ovggt.h - C ABI of the B200 streaming global-attention step of OVGGT.
+ *
+ * One handle (ovggt_cache) holds the bounded KV caches of all global-attention
+ * layers of one frame stream.  For every incoming frame and every layer the
+ * caller runs one step:
+ *
+ *   append  K_t, V_t to the layer's cache                           (Eq. 2)
+ *   attend  the frame's queries over [cache of frame t-1 ; frame t] (Sec. 3.1)
+ *   score   new tokens by FFN-residual norm, smoothed               (Eq. 5, Eq. 6)
+ *           cached tokens by key diversity, hybrid-normalised       (Eq. 7)
+ *   protect first-frame tokens and historical anchors (FIFO)        (Sec. 3.3)
+ *   select  P u Top-k(U, B - |P|) and compact the cache             (Eq. 8)
+ *
+ * Conventions
+ *  - Every `device` pointer is CUDA device memory of the GPU that was current at
+ *    ovggt_cache_create; every `host` pointer is ordinary host memory.
+ *  - Row-major, token-major tensors: [tokens, C] with C = n_heads * head_dim and head h
+ *    owning columns [h*head_dim, (h+1)*head_dim).  Element type is the configured
+ *    dtype (float, or bfloat16 bit patterns).  Tensors must be 16-byte aligned.
+ *  - Tokens of a frame: n_special aux tokens (camera, registers) first, then the
+ *    grid_h x grid_w patch tokens row-major; M = n_special + grid_h * grid_w.
+ *  - The caller owns every device byte: inputs, outputs and the workspace.  The
+ *    library never allocates or frees device memory and keeps no pointer of an
+ *    ovggt_frame_io after the call returns.  The handle itself is host memory.
+ *  - Every call enqueues its kernels on the given CUDA stream (a cudaStream_t passed
+ *    as void*; NULL = the legacy default stream) and returns without synchronising,
+ *    unless stated.  All layers of a handle share scratch memory, so all calls on one
+ *    handle must be ordered on one stream (or otherwise serialised by the caller).
+ *  - Return value: 0 on success, a negative OVGGT_ERR_* otherwise; no call aborts,
+ *    throws or prints.  A handle is not thread-safe; independent handles are independent.
+ */
+#ifndef OVGGT_H_
+#define OVGGT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define OVGGT_MAX_ANCHORS 16
+
+enum {
+  OVGGT_OK = 0,
+  OVGGT_ERR_INVALID_ARG = -1,       /* NULL handle / pointer, non-positive size, unsupported head_dim or dtype */
+  OVGGT_ERR_BAD_LAYER = -2,
+  OVGGT_ERR_BUDGET_TOO_SMALL = -3,  /* B < M, or B below the protected-set bound M + K_max * A of Eq. 9 */
+  OVGGT_ERR_FRAME_ORDER = -4,       /* frame ids must increase; attend/compress must alternate per layer */
+  OVGGT_ERR_MISALIGNED = -5,        /* a device tensor or the workspace is not 16-byte (workspace: 1024-byte) aligned */
+  OVGGT_ERR_WORKSPACE_TOO_SMALL = -6,
+  OVGGT_ERR_CUDA = -7,              /* a CUDA runtime / driver call failed; see ovggt_last_cuda_error */
+  OVGGT_ERR_DEVICE_STATUS = -8,     /* a kernel reported an inconsistency through the device status word */
+  OVGGT_ERR_TIMEOUT = -9,           /* a bounded device-side wait ran out (the kernel returned cleanly) */
+  OVGGT_ERR_UNSUPPORTED = -10       /* the configuration is valid but this build has no kernel for it */
+};
+
+enum { OVGGT_DTYPE_F32 = 0, OVGGT_DTYPE_BF16 = 1 };
+enum { OVGGT_SCORE_HYBRID = 0, OVGGT_SCORE_RESIDUAL_STORED = 1 };
+enum { OVGGT_FLAG_EVICTABLE = 0, OVGGT_FLAG_INIT = 1, OVGGT_FLAG_HIST = 2 };
+
+typedef struct ovggt_cache ovggt_cache; /* opaque host-side handle */
+
+typedef struct {
+  int32_t n_layers, n_heads, head_dim;   /* head_dim must be 64 */
+  int32_t n_special, grid_h, grid_w;     /* per-frame token layout (Sec. 3.1) */
+  const int32_t* budget;                 /* host [n_layers]: B^(l), tokens kept per layer between steps (Eq. 8) */
+  int32_t anchor_tokens;                 /* A = ceil(eta * N_p): protected patch tokens per historical anchor */
+  int32_t k_max;                         /* K_max active historical anchors, <= OVGGT_MAX_ANCHORS */
+  int32_t min_anchor_interval;           /* frames between anchor registrations (paper: 100) */
+  float tau, alpha, beta;                /* coverage threshold, smoothing strength (Eq. 6), hybrid balance (Eq. 7) */
+  int32_t protect_first_frame;           /* 1: Global Initial Anchor (all M first-frame tokens kept for good) */
+  int32_t score_mode;                    /* OVGGT_SCORE_HYBRID (Eq. 7) or OVGGT_SCORE_RESIDUAL_STORED */
+  int32_t dtype;                         /* OVGGT_DTYPE_* of q, k, v, resid, out and of the cache */
+  void* workspace;                       /* device, >= ovggt_workspace_bytes(cfg), 1024-byte aligned; need not be zeroed */
+  size_t workspace_bytes;
+} ovggt_config;
+
+typedef struct {
+  int64_t frame_id;             /* strictly increasing over the stream; the same for all layers of a frame */
+  const void* q;                /* [M, C] queries of the frame                     (attend) */
+  const void* k;                /* [M, C] keys of the frame                        (attend) */
+  const void* v;                /* [M, C] values of the frame                      (attend) */
+  const void* resid;            /* [M, C] FFN residual rows, LayerScale included   (compress, Eq. 5) */
+  const float* conf;            /* [grid_h*grid_w] per-patch confidence, or NULL = no anchor candidate (compress) */
+  float rho;                    /* coverage ratio of the latest anchor in this view; NaN = no decision (compress) */
+  const float* score_override;  /* [n + M] fp32 or NULL: priorities the selection ranks instead of its own (compress) */
+  void* out;                    /* [M, C] attention output                         (attend) */
+} ovggt_frame_io;               /* ovggt_layer_step: all pointers device.  ovggt_layer_step_host: all pointers host. */
+
+typedef struct {
+  int32_t n_cached;             /* rows held after the last completed step, <= budget */
+  int32_t n_protected_init;     /* |P_init| */
+  int32_t n_protected_hist;     /* |P_hist| = anchor_tokens * n_active_anchors */
+  int32_t n_active_anchors;
+  int64_t anchor_frames[OVGGT_MAX_ANCHORS]; /* active historical anchors, oldest first */
+  int64_t frames_seen;          /* steps completed on this layer */
+  int64_t evicted_total;        /* rows dropped so far */
+  int32_t last_n_candidates;    /* N = n + M of the last step */
+  int32_t last_n_survivors;     /* min(N, B) */
+  uint64_t bytes_resident;      /* workspace bytes this layer's K/V buffers occupy: constant over the stream */
+  int32_t device_status;        /* 0, or the OVGGT_ERR_* a kernel raised */
+} ovggt_stats;
+
+/* Bytes of device workspace the configuration needs (0 if the configuration is invalid).
+ * cfg->workspace / workspace_bytes are ignored here. */
+size_t ovggt_workspace_bytes(const ovggt_config* cfg);
+
+/* Validate cfg, lay the caches out in cfg->workspace and return a handle.  Enqueues one
+ * small clearing kernel on the legacy default stream and synchronises it.
+ * OVGGT_ERR_BUDGET_TOO_SMALL if a layer's budget cannot hold the protected set (Eq. 9). */
+int ovggt_cache_create(const ovggt_config* cfg, ovggt_cache** out);
+int ovggt_cache_destroy(ovggt_cache* cache);
+
+/* Eq. 2 + attention: append io->k / io->v as rows [n, n+M) of the layer's cache, then write
+ * softmax(Q K^T / sqrt(head_dim)) V over all n + M rows to io->out.  No mask inside the step
+ * (causality is between frames).  Uses frame_id, q, k, v, out. */
+int ovggt_layer_attend(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
+
+/* Eq. 5-8 and Sec. 3.3 for the frame appended by the last ovggt_layer_attend of this layer:
+ * score, protect, select the survivors and compact the cache to <= B^(l) rows, order preserved.
+ * The anchor decision of a frame is taken once (first layer that compresses it) from rho and the
+ * interval rule and applied identically to every layer.  Uses frame_id, resid, conf, rho,
+ * score_override. */
+int ovggt_layer_compress(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
+
+/* ovggt_layer_attend followed by ovggt_layer_compress: the whole hot path of one (frame, layer). */
+int ovggt_layer_step(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
+
+/* The same step with HOST tensors: q, k, v, resid, conf, out are host pointers (pinned memory
+ * makes the copies asynchronous); score_override must be NULL.  The inputs are copied into staging
+ * buffers of the workspace, the step runs, and out is copied back, all on `stream`.  The call returns
+ * without synchronising: out is valid once the stream has been synchronised. */
+int ovggt_layer_step_host(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
+
+/* Counters of one layer.  Synchronises the stream the handle last used (to read the device status word). */
+int ovggt_cache_stats(ovggt_cache* cache, int32_t layer, ovggt_stats* out);
+
+/* Copy the layer's current layout to host arrays, ascending token id = ascending row.  Any pointer may be
+ * NULL.  token_ids [n] (frame_id * M + index in frame), flags [n] (OVGGT_FLAG_*), scores [n] (the smoothed
+ * activation score each row had when it was new), k and v [n, C] in the configured dtype.  Synchronises. */
+int ovggt_cache_export(ovggt_cache* cache, int32_t layer, int64_t* token_ids, uint8_t* flags,
+                       float* scores, void* k, void* v, int32_t* n);
+
+/* Replace the layer's content by n rows given as host arrays (ascending token ids).  Anchor bookkeeping is
+ * rebuilt from the flags and ids; next_frame_id is the smallest frame id the stream may continue with.
+ * Synchronises. */
+int ovggt_cache_import(ovggt_cache* cache, int32_t layer, const int64_t* token_ids, const uint8_t* flags,
+                       const float* scores, const void* k, const void* v, int32_t n,
+                       int64_t next_frame_id, int64_t last_registration_frame);
+
+/* Results of the layer's last compress, copied to host (each pointer may be NULL): priorities [N] as the
+ * library computed them (+inf on protected rows; its own values even when score_override was ranked instead),
+ * survivor positions [n'] ascending, and their counts.  Synchronises. */
+int ovggt_cache_last_selection(ovggt_cache* cache, int32_t layer, float* priorities, int32_t* n_candidates,
+                               int32_t* survivors, int32_t* n_survivors);
+
+/* Per-kernel-class device time.  While enabled, every step records a pair of CUDA events (host objects, no
+ * device memory) around the launches of each class on the step's stream; the events add a little latency, so
+ * throughput is measured with profiling off.  ovggt_cache_profile_read synchronises, adds up the elapsed
+ * milliseconds and launch-group counts per class into ms / counts [OVGGT_PROF_CLASSES] (each may be NULL) and,
+ * if reset is non-zero, clears the totals. */
+enum {
+  OVGGT_PROF_APPEND = 0,     /* Eq. 2 copy of K_t, V_t */
+  OVGGT_PROF_ATTENTION = 1,  /* attention kernel and, when the KV range is split, its merge kernel */
+  OVGGT_PROF_ROW_NORMS = 2,  /* Eq. 5 */
+  OVGGT_PROF_DIVERSITY = 3,  /* key column sums + diversity */
+  OVGGT_PROF_SELECT = 4,     /* flags, Eq. 6, Eq. 7, Eq. 8 */
+  OVGGT_PROF_COMPACT = 5,    /* gather of the surviving K/V rows */
+  OVGGT_PROF_CLASSES = 6
+};
+int ovggt_cache_profile_enable(ovggt_cache* cache, int32_t enable);
+int ovggt_cache_profile_read(ovggt_cache* cache, double* ms, int64_t* counts, int32_t reset);
+
+/* Number of kernels this library has launched since it was loaded (all handles). */
+uint64_t ovggt_kernel_launches(void);
+
+const char* ovggt_strerror(int code);
+/* The cudaError_t / CUresult of the last failed CUDA call in this process (0 if none). */
+int ovggt_last_cuda_error(void);
+
+/* ------------------------------------------------------------------------------------------------
+ * Single kernels, exposed for unit parity tests and scaled micro-benchmarks.  All pointers device,
+ * dtype = OVGGT_DTYPE_*, asynchronous on `stream`.
+ * ---------------------------------------------------------------------------------------------- */
+
+/* Eq. 5: s[j] = ||x[j, :]||_2 for rows of x [rows, C]; fp32 accumulation in a fixed order. */
+int ovggt_k_row_norms(const void* x, int32_t rows, int32_t C, int32_t dtype, float* s, void* stream);
+
+/* Sec. 3.2 (Hybrid Scoring): d[i] = 1 - cos(K[i, :], sum of all rows of K) for K [rows, C].
+ * scratch: device, >= ovggt_k_diversity_scratch_bytes(rows, C). */
+size_t ovggt_k_diversity_scratch_bytes(int32_t rows, int32_t C);
+int ovggt_k_diversity(const void* K, int32_t rows, int32_t C, int32_t dtype, float* d, void* scratch,
+                      void* stream);
+
+/* Eq. 8: survivors of N candidates with priorities r [N] and flags [N] (non-zero = protected) under budget B:
+ * every protected row plus the B - |P| evictable rows of largest r, ties to the lower position, NaN ranks
+ * with -inf.  survivors [min(N, B)] ascending.  scratch: device, >= 4 * N + 64 bytes.
+ * `batch` independent problems are laid out back to back (r, flags, survivors strides N, N, B); one CTA each. */
+int ovggt_k_select(const float* r, const uint8_t* flags, int32_t N, int32_t B, int32_t batch,
+                   int32_t* survivors, void* scratch, void* stream);
+
+/* Order-preserving compaction: dst[j, :] = src[survivors[j], :] for K and V, j < n_keep. */
+int ovggt_k_compact(const void* k_src, const void* v_src, const int32_t* survivors, int32_t n_keep, int32_t C,
+                    int32_t dtype, void* k_dst, void* v_dst, void* stream);
+
+/* out [M, C] = softmax(Q K^T / sqrt(64)) V per head over N rows; head_dim 64.  bf16: tcgen05 kernel;
+ * fp32: SIMT kernel.  scratch: device, >= ovggt_k_attention_scratch_bytes(M, N, n_heads). */
+size_t ovggt_k_attention_scratch_bytes(int32_t M, int32_t N, int32_t n_heads);
+int ovggt_k_attention(const void* q, const void* k, const void* v, int32_t M, int32_t N, int32_t n_heads,
+                      int32_t dtype, void* out, void* scratch, int32_t* device_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

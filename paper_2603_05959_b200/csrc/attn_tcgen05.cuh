@@ -1,0 +1,533 @@
+// bf16 flash attention for sm_100a: out = softmax(Q K^T / sqrt(64)) V per head, head_dim 64, no mask.
+//
+// One CTA owns one 128-row query tile of one head and a contiguous range of 128-row KV tiles.
+//   warp 0      TMA producer: Q once, then K and V tiles into 128-byte-swizzled shared-memory stages
+//   warp 1      allocates tensor memory and issues tcgen05.mma:  S = Q K^T  (SS, fp32 in TMEM),
+//               O += P V (P read from TMEM as the A operand, V MN-major from shared memory)
+//   warps 2-5   softmax: one thread per query row reads its S row with tcgen05.ld, keeps a running
+//               reference maximum (rescaling O only when the maximum grows by more than 2^8), writes
+//               P as bf16 over the S columns, and at the end normalises and stores O
+// Two CTAs are resident per SM (256 TMEM columns and ~82 KB shared memory each), so one CTA's MMAs
+// overlap the other's exponentials.  The KV range may be split across CTAs; partial (O, max, sum)
+// triples are merged by a second kernel.  Every mbarrier wait is bounded: on expiry the CTA records
+// OVGGT_ERR_TIMEOUT in the status word and leaves through the common teardown.
+#pragma once
+
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace ovggt {
+
+constexpr int kBM = 128;            // query rows per CTA
+constexpr int kBN = 128;            // KV rows per tile
+constexpr int kHD = 64;             // head dim
+constexpr int kKVStages = 2;
+constexpr int kAttnThreads = 192;
+constexpr int kTileBytes = kBN * kHD * 2;          // 16 KB
+constexpr int kTmemCols = 256;
+constexpr int kColS = 0, kColO = 128;
+constexpr float kRescaleThreshold = 8.0f;          // log2 units
+constexpr int kMaxSplits = 16;
+
+struct AttnBarriers {
+  unsigned long long q_full, s_full, p_full, o_full, drain;
+  unsigned long long k_full[kKVStages], k_empty[kKVStages], v_full[kKVStages], v_empty[kKVStages];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+constexpr size_t kAttnSmemBytes = 1024 + (size_t)kTileBytes * (1 + 2 * kKVStages) + sizeof(AttnBarriers) + 64;
+
+// ---------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(void* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(void* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(void* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Wait for the phase with the given parity, for at most about one second.
+__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, AttnBarriers* B, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  unsigned long long t0 = 0;
+  for (uint32_t spins = 1;; ++spins) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((spins & 1023u) == 0) {
+      if (*(volatile int*)&B->abort_flag) return false;
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > 1000000000ull) {
+        *(volatile int*)&B->abort_flag = 1;
+        atomicCAS(status, 0, OVGGT_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int x, int y, void* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(void* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+
+// Shared-memory matrix descriptor for a 128-byte-swizzled tile whose 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)1 << 16;                  // leading byte offset (unused for one swizzle atom): 16 B
+  d |= (uint64_t)(1024 >> 4) << 32;        // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                  // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                  // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128.
+__host__ __device__ constexpr uint32_t idesc_bf16(int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(128 >> 4) << 24);
+}
+
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(d_tmem), "l"(a_desc), "l"(b_desc),
+      "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n" ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc),
+      "r"(idesc), "r"(acc)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+      "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+      "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+
+// ---------------------------------------------------------------- the kernel
+
+struct AttnParams {
+  int M, N, H;
+  int splits, tiles_per_split, tiles_total;
+  __nv_bfloat16* out;     // [M, C]            (splits == 1)
+  float* o_part;          // [splits, M, C]    un-normalised partial outputs
+  float2* ml_part;        // [splits, M, H]    (reference maximum in log2 units, row sum)
+  int* status;
+};
+
+__global__ void __launch_bounds__(kAttnThreads, 2)
+k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+               const __grid_constant__ CUtensorMap tm_v, const AttnParams P) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  unsigned char* sQ = smem;
+  unsigned char* sK = sQ + kTileBytes;
+  unsigned char* sV = sK + kKVStages * kTileBytes;
+  AttnBarriers* B = reinterpret_cast<AttnBarriers*>(sV + kKVStages * kTileBytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qt = blockIdx.x, h = blockIdx.y, split = blockIdx.z;
+  const int t_begin = split * P.tiles_per_split;
+  const int n_tiles = min(P.tiles_total, t_begin + P.tiles_per_split) - t_begin;   // >= 1 by construction
+  const int C = P.H * kHD;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&B->q_full, 1);
+    mbar_init(&B->s_full, 1);
+    mbar_init(&B->p_full, 128);
+    mbar_init(&B->o_full, 1);
+    mbar_init(&B->drain, 1);
+    for (int s = 0; s < kKVStages; ++s) {
+      mbar_init(&B->k_full[s], 1);
+      mbar_init(&B->k_empty[s], 1);
+      mbar_init(&B->v_full[s], 1);
+      mbar_init(&B->v_empty[s], 1);
+    }
+    B->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&B->tmem_base)),
+                 "r"((uint32_t)kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *(volatile uint32_t*)&B->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int issued_k = 0, issued_v = 0;
+      bool ok = true;
+      mbar_expect_tx(&B->q_full, kTileBytes);
+      tma_load_2d(sQ, &tm_q, h * kHD, qt * kBM, &B->q_full);
+      for (int it = 0; it < n_tiles && ok; ++it) {
+        const int s = it % kKVStages;
+        const uint32_t ph = (uint32_t)(it / kKVStages) & 1u;
+        const int row = (t_begin + it) * kBN;
+        ok = mbar_wait(&B->k_empty[s], ph ^ 1u, B, P.status);
+        if (!ok) break;
+        mbar_expect_tx(&B->k_full[s], kTileBytes);
+        tma_load_2d(sK + s * kTileBytes, &tm_k, h * kHD, row, &B->k_full[s]);
+        ++issued_k;
+        ok = mbar_wait(&B->v_empty[s], ph ^ 1u, B, P.status);
+        if (!ok) break;
+        mbar_expect_tx(&B->v_full[s], kTileBytes);
+        tma_load_2d(sV + s * kTileBytes, &tm_v, h * kHD, row, &B->v_full[s]);
+        ++issued_v;
+      }
+      if (!ok) {
+        // leave no bulk copy in flight into this CTA's shared memory
+        mbar_wait(&B->q_full, 0, B, P.status);
+        for (int i = max(0, issued_k - kKVStages); i < issued_k; ++i)
+          mbar_wait(&B->k_full[i % kKVStages], (uint32_t)(i / kKVStages) & 1u, B, P.status);
+        for (int i = max(0, issued_v - kKVStages); i < issued_v; ++i)
+          mbar_wait(&B->v_full[i % kKVStages], (uint32_t)(i / kKVStages) & 1u, B, P.status);
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = idesc_bf16(kBN, false);
+      constexpr uint32_t idesc_pv = idesc_bf16(kHD, true);
+      const uint64_t dq = smem_desc_sw128(smem_u32(sQ));
+      bool ok = mbar_wait(&B->q_full, 0, B, P.status);
+      for (int it = 0; it < n_tiles && ok; ++it) {
+        const int s = it % kKVStages;
+        const uint32_t ph = (uint32_t)(it / kKVStages) & 1u;
+        ok = mbar_wait(&B->k_full[s], ph, B, P.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t dk = smem_desc_sw128(smem_u32(sK + s * kTileBytes));
+#pragma unroll
+        for (int kk = 0; kk < kHD / 16; ++kk)     // 16 elements of head dim = 32 bytes inside the swizzled row
+          mma_ss(tmem + kColS, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_qk, kk > 0);
+        tc_commit(&B->k_empty[s]);
+        tc_commit(&B->s_full);
+        ok = mbar_wait(&B->p_full, (uint32_t)it & 1u, B, P.status);
+        if (!ok) break;
+        ok = mbar_wait(&B->v_full[s], ph, B, P.status);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t dv = smem_desc_sw128(smem_u32(sV + s * kTileBytes));
+#pragma unroll
+        for (int kk = 0; kk < kBN / 16; ++kk)     // 16 KV rows = 2048 bytes; P: 8 TMEM columns per 16 bf16
+          mma_ts(tmem + kColO, tmem + kColS + kk * 8, dv + (uint64_t)(kk * 128), idesc_pv, (it > 0 || kk > 0));
+        tc_commit(&B->v_empty[s]);
+      }
+      if (ok) {
+        tc_commit(&B->o_full);
+        mbar_wait(&B->o_full, 0, B, P.status);
+      } else {
+        tc_commit(&B->drain);                     // let every issued MMA finish before TMEM is freed
+        mbar_wait(&B->drain, 0, B, P.status);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------ softmax, correction and epilogue (128 threads)
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16);
+    const float c = 1.4426950408889634f * 0.125f;     // log2(e) / sqrt(64)
+    float mref = 0.0f, l = 0.0f;
+    bool ok = true;
+    for (int it = 0; it < n_tiles; ++it) {
+      ok = mbar_wait(&B->s_full, (uint32_t)it & 1u, B, P.status);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t s[128];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) tmem_ld32(t_row + kColS + j * 32, s + j * 32);
+      tmem_wait_ld();
+      const int col0 = (t_begin + it) * kBN;
+      if (col0 + kBN > P.N) {
+#pragma unroll
+        for (int j = 0; j < 128; ++j)
+          if (col0 + j >= P.N) s[j] = 0xFF800000u;     // -inf on columns past the last row
+      }
+      float mx = __uint_as_float(s[0]);
+#pragma unroll
+      for (int j = 1; j < 128; ++j) mx = fmaxf(mx, __uint_as_float(s[j]));
+      mx *= c;
+      if (it == 0) {
+        mref = mx;
+      } else {
+        const bool grow = mx - mref > kRescaleThreshold;
+        if (__any_sync(0xFFFFFFFFu, grow)) {
+          const float a = grow ? ex2(mref - mx) : 1.0f;
+          if (grow) {
+            mref = mx;
+            l *= a;
+          }
+          uint32_t o[32];
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            tmem_ld32(t_row + kColO + j * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * a);
+            tmem_st32(t_row + kColO + j * 32, o);
+          }
+        }
+      }
+      const float nm = -mref;
+      float sum = 0.0f;
+#pragma unroll
+      for (int j = 0; j < 128; j += 2) {
+        const float p0 = ex2(fmaf(__uint_as_float(s[j]), c, nm));
+        const float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), c, nm));
+        sum += p0;
+        sum += p1;
+        s[j >> 1] = pack_bf16(p0, p1);
+      }
+      l += sum;
+      tmem_st32(t_row + kColS, s);
+      tmem_st32(t_row + kColS + 32, s + 32);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&B->p_full);
+    }
+    if (ok) ok = mbar_wait(&B->o_full, 0, B, P.status);
+    if (ok) {
+      tc_fence_after();
+      const int m = qt * kBM + row;
+      const float inv = 1.0f / l;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        uint32_t o[32];
+        tmem_ld32(t_row + kColO + j * 32, o);
+        tmem_wait_ld();
+        if (m < P.M) {
+          if (P.splits == 1) {
+            uint4* dst = reinterpret_cast<uint4*>(P.out + (size_t)m * C + (size_t)h * kHD + j * 32);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              uint4 w;
+              w.x = pack_bf16(__uint_as_float(o[8 * e + 0]) * inv, __uint_as_float(o[8 * e + 1]) * inv);
+              w.y = pack_bf16(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv);
+              w.z = pack_bf16(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv);
+              w.w = pack_bf16(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv);
+              dst[e] = w;
+            }
+          } else {
+            uint4* dst = reinterpret_cast<uint4*>(P.o_part + ((size_t)split * P.M + m) * C + (size_t)h * kHD + j * 32);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) dst[e] = make_uint4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
+          }
+        }
+      }
+      if (P.splits > 1 && m < P.M) P.ml_part[((size_t)split * P.M + m) * P.H + h] = make_float2(mref, l);
+    }
+  }
+
+  // ------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols) : "memory");
+  }
+}
+
+// out[m, h*64 + c] = sum_s O_s 2^(m_s - m*) / sum_s l_s 2^(m_s - m*), m* = max_s m_s.  One thread per 4 columns.
+__global__ void __launch_bounds__(256) k_attn_merge(const float* __restrict__ o_part, const float2* __restrict__ ml_part,
+                                                    int M, int H, int splits, __nv_bfloat16* __restrict__ out) {
+  const int C = H * kHD;
+  const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t total = (size_t)M * (C / 4);
+  if (idx >= total) return;
+  const int m = (int)(idx / (C / 4)), c4 = (int)(idx % (C / 4)), h = (c4 * 4) / kHD;
+  float mstar = -INFINITY;
+  for (int s = 0; s < splits; ++s) mstar = fmaxf(mstar, ml_part[((size_t)s * M + m) * H + h].x);
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float den = 0.0f;
+  for (int s = 0; s < splits; ++s) {
+    const float2 ml = ml_part[((size_t)s * M + m) * H + h];
+    const float w = exp2f(ml.x - mstar);
+    const float4 o = *reinterpret_cast<const float4*>(o_part + ((size_t)s * M + m) * C + c4 * 4);
+    acc.x = fmaf(w, o.x, acc.x);
+    acc.y = fmaf(w, o.y, acc.y);
+    acc.z = fmaf(w, o.z, acc.z);
+    acc.w = fmaf(w, o.w, acc.w);
+    den = fmaf(w, ml.y, den);
+  }
+  const float inv = 1.0f / den;
+  uint2 w;
+  w.x = pack_bf16(acc.x * inv, acc.y * inv);
+  w.y = pack_bf16(acc.z * inv, acc.w * inv);
+  *reinterpret_cast<uint2*>(out + (size_t)m * C + c4 * 4) = w;
+}
+
+// ---------------------------------------------------------------- host side
+
+inline int g_attn_last_error = 0;
+inline int attn_tcgen05_last_error() { return g_attn_last_error; }
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// [rows, C] bf16 row-major; box = 64 columns x 128 rows, 128-byte swizzle, zero fill outside.
+inline int make_rows_map(CUtensorMap* map, const void* base, int rows, int C) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return OVGGT_ERR_CUDA;
+  cuuint64_t dims[2] = {(cuuint64_t)C, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)C * 2};
+  cuuint32_t box[2] = {kHD, kBN};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    g_attn_last_error = (int)r;
+    return OVGGT_ERR_CUDA;
+  }
+  return OVGGT_OK;
+}
+
+// Number of KV splits: minimise (waves of CTAs over 2 x 148 slots) x (tiles per CTA + fixed overhead).
+inline int attn_choose_splits(int M, int N, int H) {
+  const int q_tiles = (M + kBM - 1) / kBM, tiles = (N + kBN - 1) / kBN;
+  const long slots = 2L * 148;
+  int best = 1;
+  long best_cost = -1;
+  for (int s = 1; s <= kMaxSplits && s <= tiles; ++s) {
+    const int per = (tiles + s - 1) / s;
+    const int eff = (tiles + per - 1) / per;
+    if (eff != s) continue;
+    const long ctas = (long)q_tiles * H * s;
+    const long waves = (ctas + slots - 1) / slots;
+    const long cost = waves * (per + 3) + (s > 1 ? 2 : 0);
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best = s;
+    }
+  }
+  return best;
+}
+
+inline size_t attn_tcgen05_scratch_bytes(int M, int N, int H) {
+  (void)N;
+  const size_t C = (size_t)H * kHD;
+  return (size_t)kMaxSplits * M * C * 4 + (size_t)kMaxSplits * M * H * 8 + 1024;
+}
+
+inline int attn_tcgen05_num_launches(int M, int N, int H) { return attn_choose_splits(M, N, H) > 1 ? 2 : 1; }
+
+inline int attn_tcgen05_launch(const void* q, const void* k, const void* v, int M, int N, int H, void* out,
+                               void* scratch, int* status, cudaStream_t st) {
+  const int C = H * kHD;
+  CUtensorMap tq, tk, tv;
+  int rc = make_rows_map(&tq, q, M, C);
+  if (rc) return rc;
+  rc = make_rows_map(&tk, k, N, C);
+  if (rc) return rc;
+  rc = make_rows_map(&tv, v, N, C);
+  if (rc) return rc;
+  AttnParams P;
+  P.M = M; P.N = N; P.H = H;
+  P.tiles_total = (N + kBN - 1) / kBN;
+  P.splits = attn_choose_splits(M, N, H);
+  P.tiles_per_split = (P.tiles_total + P.splits - 1) / P.splits;
+  P.out = static_cast<__nv_bfloat16*>(out);
+  P.o_part = static_cast<float*>(scratch);
+  P.ml_part = reinterpret_cast<float2*>(static_cast<char*>(scratch) + (size_t)kMaxSplits * M * C * 4);
+  P.status = status;
+  cudaError_t e = cudaFuncSetAttribute(k_attn_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
+  if (e != cudaSuccess) { g_attn_last_error = (int)e; return OVGGT_ERR_CUDA; }
+  dim3 grid((M + kBM - 1) / kBM, H, P.splits);
+  k_attn_tcgen05<<<grid, kAttnThreads, kAttnSmemBytes, st>>>(tq, tk, tv, P);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) { g_attn_last_error = (int)e; return OVGGT_ERR_CUDA; }
+  if (P.splits > 1) {
+    const size_t total = (size_t)M * (C / 4);
+    k_attn_merge<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(P.o_part, P.ml_part, M, H, P.splits, P.out);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { g_attn_last_error = (int)e; return OVGGT_ERR_CUDA; }
+  }
+  return OVGGT_OK;
+}
+
+}  // namespace ovggt

@@ -1,0 +1,714 @@
+// Host side of the C ABI declared in include/ovggt.h: handle, bookkeeping that needs no device
+// read-back (row counts, anchor FIFO, trigger rule), workspace layout and kernel launches.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <deque>
+#include <new>
+#include <vector>
+
+#include "../../include/ovggt.h"
+#include "attn_simt.cuh"
+#include "attn_tcgen05.cuh"
+#include "common.cuh"
+#include "compact_kernels.cuh"
+#include "score_kernels.cuh"
+#include "select_kernel.cuh"
+
+using namespace ovggt;
+
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+std::atomic<int> g_last_cuda_error{0};
+
+inline int cuda_fail(cudaError_t e) {
+  g_last_cuda_error.store((int)e);
+  return OVGGT_ERR_CUDA;
+}
+#define CK(expr)                                  \
+  do {                                            \
+    cudaError_t e__ = (expr);                     \
+    if (e__ != cudaSuccess) return cuda_fail(e__); \
+  } while (0)
+#define LAUNCHED()                                 \
+  do {                                             \
+    g_launches.fetch_add(1);                       \
+    cudaError_t e__ = cudaGetLastError();          \
+    if (e__ != cudaSuccess) return cuda_fail(e__); \
+  } while (0)
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+constexpr int kMaxColsumParts = 592;       // 4 CTAs per SM on 148 SMs
+constexpr size_t kSmemLimit = 227 * 1024;
+
+int colsum_parts(int rows) { return std::max(1, std::min(kMaxColsumParts, (rows + 15) / 16)); }
+
+size_t select_smem_bytes(int N, int M, bool keys_in_smem) {
+  size_t b = align_up(sizeof(SelectShared), 16) + align_up((size_t)M * 4, 16) + (size_t)N;
+  if (keys_in_smem) b += (size_t)N * 4;
+  return b + 16;
+}
+
+// ------------------------------------------------------------------ single-kernel launchers
+
+int launch_row_norms(const void* x, int rows, int C, int dtype, float* s, cudaStream_t st) {
+  if (rows <= 0) return OVGGT_OK;
+  const int nvec = C * elem_bytes(dtype) / 16;
+  const int grid = (rows + 7) / 8;
+  if (dtype == kBF16) k_row_norms<kBF16><<<grid, 256, 0, st>>>((const uint4*)x, rows, nvec, s);
+  else                k_row_norms<kF32><<<grid, 256, 0, st>>>((const uint4*)x, rows, nvec, s);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
+// part: [colsum_parts(rows), C] floats; ksum: [C] floats.
+int launch_diversity(const void* K, int rows, int C, int dtype, float* part, float* ksum, float* d,
+                     cudaStream_t st) {
+  if (rows <= 0) return OVGGT_OK;
+  const int nvec = C * elem_bytes(dtype) / 16;
+  const int parts = colsum_parts(rows);
+  const int rpc = (rows + parts - 1) / parts;
+  const int threads = std::min(256, (nvec + 31) / 32 * 32);
+  if (dtype == kBF16) k_colsum_partial<kBF16><<<parts, threads, 0, st>>>((const uint4*)K, rows, nvec, rpc, part);
+  else                k_colsum_partial<kF32><<<parts, threads, 0, st>>>((const uint4*)K, rows, nvec, rpc, part);
+  LAUNCHED();
+  k_colsum_final<<<(C + 31) / 32, 1024, 0, st>>>(part, parts, C, ksum);
+  LAUNCHED();
+  const int grid = std::min((rows + 7) / 8, 148 * 8);
+  const size_t smem = (size_t)C * 4;
+  if (dtype == kBF16) k_diversity<kBF16><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, d);
+  else                k_diversity<kF32><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, d);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
+int launch_compact(const void* ks, const void* vs, const int* surv, int n_keep, int C, int dtype, void* kd,
+                   void* vd, cudaStream_t st) {
+  if (n_keep <= 0) return OVGGT_OK;
+  const int nvec = C * elem_bytes(dtype) / 16;
+  const int grid = std::min((2 * n_keep + 7) / 8, 148 * 8);
+  k_compact<<<grid, 256, 0, st>>>((const uint4*)ks, (const uint4*)vs, surv, n_keep, nvec, (uint4*)kd, (uint4*)vd);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
+int launch_attention(const void* q, const void* k, const void* v, int M, int N, int H, int dtype, void* out,
+                     void* scratch, int* status, cudaStream_t st) {
+  if (dtype == kBF16) {
+    int rc = attn_tcgen05_launch(q, k, v, M, N, H, out, scratch, status, st);
+    if (rc == OVGGT_OK) g_launches.fetch_add(attn_tcgen05_num_launches(M, N, H));
+    if (rc == OVGGT_ERR_CUDA) g_last_cuda_error.store(attn_tcgen05_last_error());
+    return rc;
+  }
+  dim3 grid((M + kSimtRows - 1) / kSimtRows, H);
+  k_attn_simt<kF32><<<grid, kSimtRows, 0, st>>>(q, k, v, M, N, H, out);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ handle
+
+struct LayerState {
+  int budget = 0;
+  int n = 0;            // rows held between steps
+  int cur = 0;          // which of the two buffers holds them
+  bool pending = false; // a frame was appended and not yet compressed
+  int64_t frames_seen = 0, evicted_total = 0, pending_frame = -1;
+  int n_prot_init = 0, n_prot_hist = 0;
+  int last_N = 0, last_keep = 0;
+  // device pointers
+  char* kbuf[2];
+  char* vbuf[2];
+  long long* ids[2];
+  uint8_t* flags[2];
+  float* stored[2];
+  float *s_raw, *d, *r;
+  int* surv;
+  uint32_t* gkeys;
+  int* n_keep_dev;
+  size_t kv_bytes = 0;
+};
+
+struct ovggt_cache {
+  ovggt_config cfg;
+  int M = 0, C = 0, Np = 0, elem = 0;
+  std::vector<int32_t> budgets;
+  std::vector<LayerState> layers;
+  // anchors (shared by all layers: the decision of a frame is taken once)
+  std::deque<int64_t> anchors;
+  int64_t first_frame = -1, last_registration = -1;
+  int64_t decided_frame = -1;
+  bool decided_register = false;
+  int64_t decided_demote = -1;
+  // shared scratch
+  float *colsum_part = nullptr, *ksum = nullptr;
+  void* attn_scratch = nullptr;
+  int* status = nullptr;
+  char *stage_q = nullptr, *stage_k = nullptr, *stage_v = nullptr, *stage_r = nullptr, *stage_o = nullptr;
+  float* stage_conf = nullptr;
+  float w_center = 0, w_edge = 0, w_corner = 0;
+  cudaStream_t last_stream = nullptr;
+  int max_rows = 0;
+  // optional per-kernel-class timing (host-side CUDA events; no device memory)
+  bool prof = false;
+  struct ProfRec { int cls; cudaEvent_t a, b; };
+  std::vector<ProfRec> prof_recs;
+  double prof_ms[OVGGT_PROF_CLASSES] = {0};
+  int64_t prof_cnt[OVGGT_PROF_CLASSES] = {0};
+};
+
+namespace {
+// Records a pair of events around the launches of one kernel class while profiling is on.
+struct ProfScope {
+  ovggt_cache* h;
+  ovggt_cache::ProfRec rec;
+  cudaStream_t st;
+  bool on;
+  ProfScope(ovggt_cache* h_, int cls, cudaStream_t st_) : h(h_), st(st_), on(h_->prof) {
+    if (!on) return;
+    rec.cls = cls;
+    if (cudaEventCreate(&rec.a) != cudaSuccess || cudaEventCreate(&rec.b) != cudaSuccess) { on = false; return; }
+    cudaEventRecord(rec.a, st);
+  }
+  ~ProfScope() {
+    if (!on) return;
+    cudaEventRecord(rec.b, st);
+    h->prof_recs.push_back(rec);
+  }
+};
+}  // namespace
+
+namespace {
+
+struct Layout {
+  size_t total = 0;
+  size_t take(size_t bytes, size_t align = 1024) {
+    total = align_up(total, align);
+    size_t off = total;
+    total += bytes;
+    return off;
+  }
+};
+
+bool config_ok(const ovggt_config* c, int* err) {
+  *err = OVGGT_ERR_INVALID_ARG;
+  if (!c || !c->budget) return false;
+  if (c->n_layers < 1 || c->n_heads < 1 || c->head_dim != 64) return false;
+  if (c->n_special < 0 || c->grid_h < 1 || c->grid_w < 1) return false;
+  if (c->anchor_tokens < 0 || c->anchor_tokens > c->grid_h * c->grid_w) return false;
+  if (c->k_max < 0 || c->k_max > OVGGT_MAX_ANCHORS || c->min_anchor_interval < 0) return false;
+  if (c->dtype != kF32 && c->dtype != kBF16) return false;
+  if (c->score_mode != OVGGT_SCORE_HYBRID && c->score_mode != OVGGT_SCORE_RESIDUAL_STORED) return false;
+  if (!(c->alpha >= 0.0f && c->alpha <= 1.0f) || !(c->beta >= 0.0f && c->beta <= 1.0f)) return false;
+  const int64_t M = c->n_special + (int64_t)c->grid_h * c->grid_w;
+  const int64_t pmax = (c->protect_first_frame ? M : 0) + (int64_t)c->k_max * c->anchor_tokens;
+  for (int l = 0; l < c->n_layers; ++l) {
+    if (c->budget[l] < M || c->budget[l] < pmax) {
+      *err = OVGGT_ERR_BUDGET_TOO_SMALL;
+      return false;
+    }
+    if ((int64_t)c->budget[l] + M > (1 << 30)) return false;
+  }
+  *err = OVGGT_OK;
+  return true;
+}
+
+// Lays the workspace out; with a handle, also records the pointers.
+size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
+  Layout L;
+  const int M = c->n_special + c->grid_h * c->grid_w, C = c->n_heads * c->head_dim;
+  const int Np = c->grid_h * c->grid_w;
+  const size_t eb = (size_t)elem_bytes(c->dtype);
+  char* base = h ? static_cast<char*>(c->workspace) : nullptr;
+  int max_rows = 0;
+  for (int l = 0; l < c->n_layers; ++l) {
+    const size_t R = (size_t)c->budget[l] + M;
+    max_rows = std::max(max_rows, (int)R);
+    size_t off[16];
+    int i = 0;
+    for (int b = 0; b < 2; ++b) off[i++] = L.take(R * C * eb);
+    for (int b = 0; b < 2; ++b) off[i++] = L.take(R * C * eb);
+    for (int b = 0; b < 2; ++b) off[i++] = L.take(R * 8);
+    for (int b = 0; b < 2; ++b) off[i++] = L.take(R);
+    for (int b = 0; b < 2; ++b) off[i++] = L.take(R * 4);
+    off[i++] = L.take((size_t)M * 4);   // s_raw
+    off[i++] = L.take(R * 4);           // d
+    off[i++] = L.take(R * 4);           // r
+    off[i++] = L.take(R * 4);           // survivors
+    off[i++] = L.take(R * 4);           // gkeys
+    off[i++] = L.take(64);              // n_keep
+    if (h) {
+      LayerState& S = h->layers[l];
+      i = 0;
+      for (int b = 0; b < 2; ++b) S.kbuf[b] = base + off[i++];
+      for (int b = 0; b < 2; ++b) S.vbuf[b] = base + off[i++];
+      for (int b = 0; b < 2; ++b) S.ids[b] = reinterpret_cast<long long*>(base + off[i++]);
+      for (int b = 0; b < 2; ++b) S.flags[b] = reinterpret_cast<uint8_t*>(base + off[i++]);
+      for (int b = 0; b < 2; ++b) S.stored[b] = reinterpret_cast<float*>(base + off[i++]);
+      S.s_raw = reinterpret_cast<float*>(base + off[i++]);
+      S.d = reinterpret_cast<float*>(base + off[i++]);
+      S.r = reinterpret_cast<float*>(base + off[i++]);
+      S.surv = reinterpret_cast<int*>(base + off[i++]);
+      S.gkeys = reinterpret_cast<uint32_t*>(base + off[i++]);
+      S.n_keep_dev = reinterpret_cast<int*>(base + off[i++]);
+      S.budget = c->budget[l];
+      S.kv_bytes = 4 * R * C * eb;
+    }
+  }
+  const size_t o_part = L.take((size_t)kMaxColsumParts * C * 4);
+  const size_t o_ksum = L.take((size_t)C * 4);
+  const size_t o_attn = L.take(ovggt_k_attention_scratch_bytes(M, max_rows, c->n_heads));
+  const size_t o_status = L.take(64);
+  size_t o_stage[5];
+  for (int i = 0; i < 5; ++i) o_stage[i] = L.take((size_t)M * C * eb);
+  const size_t o_conf = L.take((size_t)Np * 4);
+  if (h) {
+    h->colsum_part = reinterpret_cast<float*>(base + o_part);
+    h->ksum = reinterpret_cast<float*>(base + o_ksum);
+    h->attn_scratch = base + o_attn;
+    h->status = reinterpret_cast<int*>(base + o_status);
+    h->stage_q = base + o_stage[0];
+    h->stage_k = base + o_stage[1];
+    h->stage_v = base + o_stage[2];
+    h->stage_r = base + o_stage[3];
+    h->stage_o = base + o_stage[4];
+    h->stage_conf = reinterpret_cast<float*>(base + o_conf);
+    h->max_rows = max_rows;
+  }
+  return align_up(L.total, 1024);
+}
+
+int check_layer(ovggt_cache* h, int32_t layer) {
+  if (!h) return OVGGT_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= (int)h->layers.size()) return OVGGT_ERR_BAD_LAYER;
+  return OVGGT_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------ exported API
+
+extern "C" size_t ovggt_workspace_bytes(const ovggt_config* cfg) {
+  int err;
+  if (!config_ok(cfg, &err)) return 0;
+  return layout_workspace(cfg, nullptr);
+}
+
+extern "C" int ovggt_cache_create(const ovggt_config* cfg, ovggt_cache** out) {
+  if (!out) return OVGGT_ERR_INVALID_ARG;
+  *out = nullptr;
+  int err;
+  if (!config_ok(cfg, &err)) return err;
+  if (!cfg->workspace) return OVGGT_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(cfg->workspace) & 1023) return OVGGT_ERR_MISALIGNED;
+  if (cfg->workspace_bytes < layout_workspace(cfg, nullptr)) return OVGGT_ERR_WORKSPACE_TOO_SMALL;
+  ovggt_cache* h = new (std::nothrow) ovggt_cache();
+  if (!h) return OVGGT_ERR_INVALID_ARG;
+  h->cfg = *cfg;
+  h->budgets.assign(cfg->budget, cfg->budget + cfg->n_layers);
+  h->cfg.budget = h->budgets.data();
+  h->M = cfg->n_special + cfg->grid_h * cfg->grid_w;
+  h->C = cfg->n_heads * cfg->head_dim;
+  h->Np = cfg->grid_h * cfg->grid_w;
+  h->elem = elem_bytes(cfg->dtype);
+  h->layers.resize(cfg->n_layers);
+  layout_workspace(&h->cfg, h);
+  // Eq. 6: 3x3 Gaussian, sigma = 1, normalised
+  const double e1 = std::exp(-0.5), e2 = std::exp(-1.0), z = 1.0 + 4.0 * e1 + 4.0 * e2;
+  h->w_center = (float)(1.0 / z);
+  h->w_edge = (float)(e1 / z);
+  h->w_corner = (float)(e2 / z);
+  cudaError_t e = cudaMemset(h->status, 0, 64);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    delete h;
+    return cuda_fail(e);
+  }
+  *out = h;
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_cache_destroy(ovggt_cache* h) {
+  if (!h) return OVGGT_ERR_INVALID_ARG;
+  for (auto& r : h->prof_recs) {
+    cudaEventDestroy(r.a);
+    cudaEventDestroy(r.b);
+  }
+  delete h;
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_layer_attend(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
+  int rc = check_layer(h, layer);
+  if (rc) return rc;
+  if (!io || !io->q || !io->k || !io->v || !io->out) return OVGGT_ERR_INVALID_ARG;
+  if (!aligned16(io->q) || !aligned16(io->k) || !aligned16(io->v) || !aligned16(io->out)) return OVGGT_ERR_MISALIGNED;
+  LayerState& S = h->layers[layer];
+  if (S.pending) return OVGGT_ERR_FRAME_ORDER;
+  if (S.frames_seen > 0 && io->frame_id <= S.pending_frame) return OVGGT_ERR_FRAME_ORDER;
+  if (io->frame_id < 0 || (h->first_frame >= 0 && io->frame_id < h->first_frame)) return OVGGT_ERR_FRAME_ORDER;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  h->last_stream = st;
+  const int M = h->M, C = h->C, nvec = C * h->elem / 16, b = S.cur;
+  const int grid = std::min((2 * M + 7) / 8, 148 * 8);
+  {
+    ProfScope ps(h, OVGGT_PROF_APPEND, st);
+    k_append<<<grid, 256, 0, st>>>((const uint4*)io->k, (const uint4*)io->v, M, nvec, S.n, (long long)io->frame_id,
+                                   (uint4*)S.kbuf[b], (uint4*)S.vbuf[b], S.ids[b], S.flags[b], S.stored[b]);
+    LAUNCHED();
+  }
+  {
+    ProfScope ps(h, OVGGT_PROF_ATTENTION, st);
+    rc = launch_attention(io->q, S.kbuf[b], S.vbuf[b], M, S.n + M, h->cfg.n_heads, h->cfg.dtype, io->out,
+                          h->attn_scratch, h->status, st);
+  }
+  if (rc) return rc;
+  if (h->first_frame < 0) {
+    h->first_frame = io->frame_id;
+    h->last_registration = io->frame_id;   // the first frame is the initial anchor
+  }
+  S.pending = true;
+  S.pending_frame = io->frame_id;
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
+  int rc = check_layer(h, layer);
+  if (rc) return rc;
+  if (!io || !io->resid) return OVGGT_ERR_INVALID_ARG;
+  if (!aligned16(io->resid)) return OVGGT_ERR_MISALIGNED;
+  LayerState& S = h->layers[layer];
+  if (!S.pending || io->frame_id != S.pending_frame) return OVGGT_ERR_FRAME_ORDER;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  h->last_stream = st;
+  const ovggt_config& c = h->cfg;
+  const int M = h->M, C = h->C, n = S.n, N = n + M, B = S.budget, b = S.cur;
+  const int64_t t = io->frame_id;
+
+  // Anchor decision of this frame (Sec. 3.3), taken once and shared by all layers.
+  if (h->decided_frame != t) {
+    h->decided_frame = t;
+    h->decided_register = false;
+    h->decided_demote = -1;
+    if (t != h->first_frame && c.anchor_tokens > 0 && c.k_max > 0 && io->conf != nullptr && io->rho < c.tau &&
+        t - h->last_registration >= c.min_anchor_interval) {
+      h->decided_register = true;
+      h->anchors.push_back(t);
+      h->last_registration = t;
+      if ((int)h->anchors.size() > c.k_max) {
+        h->decided_demote = h->anchors.front();
+        h->anchors.pop_front();
+      }
+    }
+  }
+  const bool first = (t == h->first_frame);
+
+  {
+    ProfScope ps(h, OVGGT_PROF_ROW_NORMS, st);
+    rc = launch_row_norms(io->resid, M, C, c.dtype, S.s_raw, st);
+  }
+  if (rc) return rc;
+  if (c.score_mode == OVGGT_SCORE_HYBRID && n > 0) {
+    ProfScope ps(h, OVGGT_PROF_DIVERSITY, st);
+    rc = launch_diversity(S.kbuf[b], n, C, c.dtype, h->colsum_part, h->ksum, S.d, st);
+    if (rc) return rc;
+  }
+  CompressParams P;
+  P.n = n; P.M = M; P.B = B;
+  P.n_special = c.n_special; P.grid_h = c.grid_h; P.grid_w = c.grid_w;
+  P.alpha = c.alpha; P.w_center = h->w_center; P.w_edge = h->w_edge; P.w_corner = h->w_corner;
+  P.beta = c.beta;
+  P.mode = c.score_mode;
+  P.protect_new = (first && c.protect_first_frame) ? 1 : 0;
+  P.register_anchor = h->decided_register ? 1 : 0;
+  P.A = c.anchor_tokens;
+  P.demote_frame = h->decided_demote;
+  P.s_raw = S.s_raw; P.d = S.d; P.conf = io->conf; P.override_r = io->score_override;
+  P.ids_src = S.ids[b]; P.flags_src = S.flags[b]; P.stored_src = S.stored[b];
+  P.ids_dst = S.ids[b ^ 1]; P.flags_dst = S.flags[b ^ 1]; P.stored_dst = S.stored[b ^ 1];
+  P.r_out = S.r; P.survivors = S.surv; P.gkeys = S.gkeys;
+  P.status = h->status; P.n_keep_out = S.n_keep_dev;
+  size_t smem = select_smem_bytes(N, M, true);
+  P.keys_in_smem = 1;
+  if (smem > kSmemLimit) {
+    P.keys_in_smem = 0;
+    smem = select_smem_bytes(N, M, false);
+    if (smem > kSmemLimit) return OVGGT_ERR_UNSUPPORTED;
+  }
+  CK(cudaFuncSetAttribute(k_compress_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit));
+  {
+    ProfScope ps(h, OVGGT_PROF_SELECT, st);
+    k_compress_select<<<1, kSelectThreads, smem, st>>>(P);
+    LAUNCHED();
+  }
+  const int n_keep = std::min(N, B);
+  {
+    ProfScope ps(h, OVGGT_PROF_COMPACT, st);
+    rc = launch_compact(S.kbuf[b], S.vbuf[b], S.surv, n_keep, C, c.dtype, S.kbuf[b ^ 1], S.vbuf[b ^ 1], st);
+  }
+  if (rc) return rc;
+
+  // bookkeeping that follows deterministically from the sizes
+  if (first && c.protect_first_frame) S.n_prot_init = M;
+  if (h->decided_register) S.n_prot_hist += c.anchor_tokens;
+  if (h->decided_demote >= 0) S.n_prot_hist -= c.anchor_tokens;
+  S.evicted_total += N - n_keep;
+  S.last_N = N;
+  S.last_keep = n_keep;
+  S.n = n_keep;
+  S.cur = b ^ 1;
+  S.pending = false;
+  S.frames_seen += 1;
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
+  int rc = ovggt_layer_attend(h, layer, io, stream);
+  if (rc) return rc;
+  return ovggt_layer_compress(h, layer, io, stream);
+}
+
+extern "C" int ovggt_layer_step_host(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
+  int rc = check_layer(h, layer);
+  if (rc) return rc;
+  if (!io || !io->q || !io->k || !io->v || !io->resid || !io->out || io->score_override) return OVGGT_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)h->M * h->C * h->elem;
+  CK(cudaMemcpyAsync(h->stage_q, io->q, bytes, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(h->stage_k, io->k, bytes, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(h->stage_v, io->v, bytes, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(h->stage_r, io->resid, bytes, cudaMemcpyHostToDevice, st));
+  if (io->conf) CK(cudaMemcpyAsync(h->stage_conf, io->conf, (size_t)h->Np * 4, cudaMemcpyHostToDevice, st));
+  ovggt_frame_io dev = *io;
+  dev.q = h->stage_q; dev.k = h->stage_k; dev.v = h->stage_v; dev.resid = h->stage_r;
+  dev.conf = io->conf ? h->stage_conf : nullptr;
+  dev.out = h->stage_o;
+  rc = ovggt_layer_step(h, layer, &dev, stream);
+  if (rc) return rc;
+  CK(cudaMemcpyAsync(io->out, h->stage_o, bytes, cudaMemcpyDeviceToHost, st));
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_cache_stats(ovggt_cache* h, int32_t layer, ovggt_stats* out) {
+  int rc = check_layer(h, layer);
+  if (rc) return rc;
+  if (!out) return OVGGT_ERR_INVALID_ARG;
+  const LayerState& S = h->layers[layer];
+  std::memset(out, 0, sizeof(*out));
+  out->n_cached = S.n;
+  out->n_protected_init = S.n_prot_init;
+  out->n_protected_hist = S.n_prot_hist;
+  out->n_active_anchors = (int)h->anchors.size();
+  int i = 0;
+  for (int64_t f : h->anchors) out->anchor_frames[i++] = f;
+  out->frames_seen = S.frames_seen;
+  out->evicted_total = S.evicted_total;
+  out->last_n_candidates = S.last_N;
+  out->last_n_survivors = S.last_keep;
+  out->bytes_resident = S.kv_bytes;
+  CK(cudaStreamSynchronize(h->last_stream));
+  int status = 0;
+  CK(cudaMemcpy(&status, h->status, sizeof(int), cudaMemcpyDeviceToHost));
+  out->device_status = status;
+  return status == 0 ? OVGGT_OK : status;
+}
+
+extern "C" int ovggt_cache_export(ovggt_cache* h, int32_t layer, int64_t* token_ids, uint8_t* flags, float* scores,
+                                  void* k, void* v, int32_t* n_out) {
+  int rc = check_layer(h, layer);
+  if (rc) return rc;
+  const LayerState& S = h->layers[layer];
+  if (S.pending) return OVGGT_ERR_FRAME_ORDER;
+  CK(cudaStreamSynchronize(h->last_stream));
+  const int n = S.n, b = S.cur;
+  const size_t row = (size_t)h->C * h->elem;
+  if (n > 0) {
+    if (token_ids) CK(cudaMemcpy(token_ids, S.ids[b], (size_t)n * 8, cudaMemcpyDeviceToHost));
+    if (flags) CK(cudaMemcpy(flags, S.flags[b], (size_t)n, cudaMemcpyDeviceToHost));
+    if (scores) CK(cudaMemcpy(scores, S.stored[b], (size_t)n * 4, cudaMemcpyDeviceToHost));
+    if (k) CK(cudaMemcpy(k, S.kbuf[b], (size_t)n * row, cudaMemcpyDeviceToHost));
+    if (v) CK(cudaMemcpy(v, S.vbuf[b], (size_t)n * row, cudaMemcpyDeviceToHost));
+  }
+  if (n_out) *n_out = n;
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_cache_import(ovggt_cache* h, int32_t layer, const int64_t* token_ids, const uint8_t* flags,
+                                  const float* scores, const void* k, const void* v, int32_t n,
+                                  int64_t next_frame_id, int64_t last_registration_frame) {
+  int rc = check_layer(h, layer);
+  if (rc) return rc;
+  LayerState& S = h->layers[layer];
+  if (n < 0 || n > S.budget || (n > 0 && (!token_ids || !flags || !scores || !k || !v))) return OVGGT_ERR_INVALID_ARG;
+  const int M = h->M;
+  // rebuild the bookkeeping from ids and flags
+  int n_init = 0, n_hist = 0;
+  std::vector<int64_t> anchor_frames;
+  for (int i = 0; i < n; ++i) {
+    if (i > 0 && token_ids[i] <= token_ids[i - 1]) return OVGGT_ERR_INVALID_ARG;
+    if (flags[i] == OVGGT_FLAG_INIT) ++n_init;
+    else if (flags[i] == OVGGT_FLAG_HIST) {
+      ++n_hist;
+      const int64_t f = token_ids[i] / M;
+      if (anchor_frames.empty() || anchor_frames.back() != f) anchor_frames.push_back(f);
+    } else if (flags[i] != OVGGT_FLAG_EVICTABLE) return OVGGT_ERR_INVALID_ARG;
+  }
+  if ((int)anchor_frames.size() > h->cfg.k_max) return OVGGT_ERR_INVALID_ARG;
+  CK(cudaStreamSynchronize(h->last_stream));
+  const int b = S.cur;
+  const size_t row = (size_t)h->C * h->elem;
+  if (n > 0) {
+    CK(cudaMemcpy(S.ids[b], token_ids, (size_t)n * 8, cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(S.flags[b], flags, (size_t)n, cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(S.stored[b], scores, (size_t)n * 4, cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(S.kbuf[b], k, (size_t)n * row, cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(S.vbuf[b], v, (size_t)n * row, cudaMemcpyHostToDevice));
+  }
+  S.n = n;
+  S.pending = false;
+  S.n_prot_init = n_init;
+  S.n_prot_hist = n_hist;
+  S.pending_frame = next_frame_id - 1;
+  S.frames_seen = n > 0 ? 1 : 0;
+  h->anchors.assign(anchor_frames.begin(), anchor_frames.end());
+  h->first_frame = n > 0 ? token_ids[0] / M : -1;
+  h->last_registration = n > 0 ? last_registration_frame : -1;
+  h->decided_frame = -1;
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_cache_last_selection(ovggt_cache* h, int32_t layer, float* priorities, int32_t* n_candidates,
+                                          int32_t* survivors, int32_t* n_survivors) {
+  int rc = check_layer(h, layer);
+  if (rc) return rc;
+  const LayerState& S = h->layers[layer];
+  CK(cudaStreamSynchronize(h->last_stream));
+  if (priorities && S.last_N > 0) CK(cudaMemcpy(priorities, S.r, (size_t)S.last_N * 4, cudaMemcpyDeviceToHost));
+  if (survivors && S.last_keep > 0) CK(cudaMemcpy(survivors, S.surv, (size_t)S.last_keep * 4, cudaMemcpyDeviceToHost));
+  if (n_candidates) *n_candidates = S.last_N;
+  if (n_survivors) *n_survivors = S.last_keep;
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_cache_profile_enable(ovggt_cache* h, int32_t enable) {
+  if (!h) return OVGGT_ERR_INVALID_ARG;
+  h->prof = enable != 0;
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_cache_profile_read(ovggt_cache* h, double* ms, int64_t* counts, int32_t reset) {
+  if (!h) return OVGGT_ERR_INVALID_ARG;
+  CK(cudaStreamSynchronize(h->last_stream));
+  for (auto& r : h->prof_recs) {
+    float t = 0.0f;
+    if (cudaEventElapsedTime(&t, r.a, r.b) == cudaSuccess) {
+      h->prof_ms[r.cls] += t;
+      h->prof_cnt[r.cls] += 1;
+    }
+    cudaEventDestroy(r.a);
+    cudaEventDestroy(r.b);
+  }
+  h->prof_recs.clear();
+  for (int i = 0; i < OVGGT_PROF_CLASSES; ++i) {
+    if (ms) ms[i] = h->prof_ms[i];
+    if (counts) counts[i] = h->prof_cnt[i];
+    if (reset) { h->prof_ms[i] = 0.0; h->prof_cnt[i] = 0; }
+  }
+  return OVGGT_OK;
+}
+
+extern "C" uint64_t ovggt_kernel_launches(void) { return g_launches.load(); }
+extern "C" int ovggt_last_cuda_error(void) { return g_last_cuda_error.load(); }
+
+extern "C" const char* ovggt_strerror(int code) {
+  switch (code) {
+    case OVGGT_OK: return "ok";
+    case OVGGT_ERR_INVALID_ARG: return "invalid argument";
+    case OVGGT_ERR_BAD_LAYER: return "layer index out of range";
+    case OVGGT_ERR_BUDGET_TOO_SMALL: return "budget below the protected-set bound M + K_max * A";
+    case OVGGT_ERR_FRAME_ORDER: return "frame ids must increase and attend/compress must alternate";
+    case OVGGT_ERR_MISALIGNED: return "pointer not sufficiently aligned";
+    case OVGGT_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case OVGGT_ERR_CUDA: return "CUDA call failed";
+    case OVGGT_ERR_DEVICE_STATUS: return "a kernel reported an inconsistency";
+    case OVGGT_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case OVGGT_ERR_UNSUPPORTED: return "configuration not supported by this build";
+    default: return "unknown error";
+  }
+}
+
+// ------------------------------------------------------------------ single kernels
+
+extern "C" int ovggt_k_row_norms(const void* x, int32_t rows, int32_t C, int32_t dtype, float* s, void* stream) {
+  if (!x || !s || rows < 0 || C < 1 || (C * elem_bytes(dtype)) % 16 || (dtype != kF32 && dtype != kBF16))
+    return OVGGT_ERR_INVALID_ARG;
+  if (!aligned16(x)) return OVGGT_ERR_MISALIGNED;
+  return launch_row_norms(x, rows, C, dtype, s, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t ovggt_k_diversity_scratch_bytes(int32_t rows, int32_t C) {
+  (void)rows;
+  return ((size_t)kMaxColsumParts + 1) * (size_t)C * 4;
+}
+
+extern "C" int ovggt_k_diversity(const void* K, int32_t rows, int32_t C, int32_t dtype, float* d, void* scratch,
+                                 void* stream) {
+  if (!K || !d || !scratch || rows < 0 || C < 1 || (C * elem_bytes(dtype)) % 16 || (dtype != kF32 && dtype != kBF16) ||
+      (size_t)C * 4 > 48 * 1024)
+    return OVGGT_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(scratch)) return OVGGT_ERR_MISALIGNED;
+  float* part = static_cast<float*>(scratch);
+  float* ksum = part + (size_t)kMaxColsumParts * C;
+  return launch_diversity(K, rows, C, dtype, part, ksum, d, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int ovggt_k_select(const float* r, const uint8_t* flags, int32_t N, int32_t B, int32_t batch,
+                              int32_t* survivors, void* scratch, void* stream) {
+  if (!r || !flags || !survivors || !scratch || N < 1 || B < 0 || batch < 1) return OVGGT_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int* status = reinterpret_cast<int*>(scratch);
+  uint32_t* gkeys = reinterpret_cast<uint32_t*>(static_cast<char*>(scratch) + 64);
+  size_t smem = align_up(sizeof(SelectShared), 16) + (size_t)N * 5 + 16;
+  int in_smem = 1;
+  if (smem > kSmemLimit || batch > 1) {
+    // batched problems keep their keys in global memory so that several CTAs fit on one SM
+    in_smem = smem <= 48 * 1024 ? 1 : 0;
+    if (!in_smem) smem = align_up(sizeof(SelectShared), 16) + (size_t)N + 16;
+    if (smem > kSmemLimit) return OVGGT_ERR_UNSUPPORTED;
+  }
+  CK(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit));
+  CK(cudaMemsetAsync(status, 0, 4, st));
+  k_select<<<batch, kSelectThreads, smem, st>>>(r, flags, N, B, survivors, gkeys, in_smem, status);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_k_compact(const void* k_src, const void* v_src, const int32_t* survivors, int32_t n_keep,
+                               int32_t C, int32_t dtype, void* k_dst, void* v_dst, void* stream) {
+  if (!k_src || !v_src || !survivors || !k_dst || !v_dst || n_keep < 0 || C < 1 || (C * elem_bytes(dtype)) % 16)
+    return OVGGT_ERR_INVALID_ARG;
+  if (!aligned16(k_src) || !aligned16(v_src) || !aligned16(k_dst) || !aligned16(v_dst)) return OVGGT_ERR_MISALIGNED;
+  return launch_compact(k_src, v_src, survivors, n_keep, C, dtype, k_dst, v_dst, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t ovggt_k_attention_scratch_bytes(int32_t M, int32_t N, int32_t n_heads) {
+  return attn_tcgen05_scratch_bytes(M, N, n_heads);
+}
+
+extern "C" int ovggt_k_attention(const void* q, const void* k, const void* v, int32_t M, int32_t N, int32_t n_heads,
+                                 int32_t dtype, void* out, void* scratch, int32_t* device_status, void* stream) {
+  if (!q || !k || !v || !out || M < 1 || N < 1 || n_heads < 1 || (dtype != kF32 && dtype != kBF16))
+    return OVGGT_ERR_INVALID_ARG;
+  if (dtype == kBF16 && (!scratch || !device_status)) return OVGGT_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return OVGGT_ERR_MISALIGNED;
+  return launch_attention(q, k, v, M, N, n_heads, dtype, out, scratch, device_status, static_cast<cudaStream_t>(stream));
+}

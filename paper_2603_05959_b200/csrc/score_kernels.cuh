@@ -1,0 +1,146 @@
+// Scoring kernels: residual norms (Eq. 5), key column sums and key diversity (Sec. 3.2).
+// All of them stream rows of [rows, C] once with 16-byte loads and accumulate in fp32 in an
+// order that depends only on the shapes, so results are reproducible run to run.
+#pragma once
+
+#include "common.cuh"
+
+namespace ovggt {
+
+// s[row] = sqrt(sum_c x[row, c]^2); one warp per row.  Lane l owns vectors l, l+32, ... and
+// folds them in that order; lanes are combined by the fixed butterfly of warp_sum.
+template <int DT>
+__global__ void __launch_bounds__(256) k_row_norms(const uint4* __restrict__ x, int rows, int nvec,
+                                                   float* __restrict__ s) {
+  constexpr int VEC = VecOf<DT>::n;
+  const int lane = threadIdx.x & 31;
+  const int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5);
+  if (row >= rows) return;
+  const uint4* p = x + (size_t)row * nvec;
+  float acc = 0.0f;
+  for (int v0 = lane; v0 < nvec; v0 += 128) {
+    uint4 u[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (v0 + 32 * i < nvec) u[i] = ld_nc(p + v0 + 32 * i);
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (v0 + 32 * i < nvec) {
+        float f[VEC];
+        unpack<DT>(u[i], f);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc = __fmaf_rn(f[e], f[e], acc);
+      }
+  }
+  acc = warp_sum(acc);
+  if (lane == 0) s[row] = __fsqrt_rn(acc);
+}
+
+// Column sums of K [rows, C], stage 1: CTA p sums its contiguous chunk of rows, in row order,
+// into part[p, C].  Thread t owns vector columns t, t + blockDim, ...
+template <int DT>
+__global__ void __launch_bounds__(256) k_colsum_partial(const uint4* __restrict__ K, int rows, int nvec,
+                                                        int rows_per_cta, float* __restrict__ part) {
+  constexpr int VEC = VecOf<DT>::n;
+  const int r0 = blockIdx.x * rows_per_cta;
+  const int r1 = min(rows, r0 + rows_per_cta);
+  for (int v = threadIdx.x; v < nvec; v += blockDim.x) {
+    float acc[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[e] = 0.0f;
+    int r = r0;
+    for (; r + 4 <= r1; r += 4) {
+      uint4 u[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) u[i] = ld_nc(K + (size_t)(r + i) * nvec + v);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float f[VEC];
+        unpack<DT>(u[i], f);
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) acc[e] += f[e];
+      }
+    }
+    for (; r < r1; ++r) {
+      float f[VEC];
+      unpack<DT>(ld_nc(K + (size_t)r * nvec + v), f);
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) acc[e] += f[e];
+    }
+    float* o = part + (size_t)blockIdx.x * nvec * VEC + (size_t)v * VEC;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) o[e] = acc[e];
+  }
+}
+
+// Stage 2: ksum[c] = sum_p part[p, c].  A CTA of 32 x 32 threads owns 32 columns; thread (py, cx)
+// folds partials py, py + 32, ... in order, then the 32 py-values are folded in order.
+__global__ void __launch_bounds__(1024) k_colsum_final(const float* __restrict__ part, int nparts, int C,
+                                                       float* __restrict__ ksum) {
+  __shared__ float sh[32][33];
+  const int cx = threadIdx.x & 31, py = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + cx;
+  float acc = 0.0f;
+  if (c < C)
+    for (int p = py; p < nparts; p += 32) acc += part[(size_t)p * C + c];
+  sh[py][cx] = acc;
+  __syncthreads();
+  if (py == 0 && c < C) {
+    float t = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) t += sh[i][cx];
+    ksum[c] = t;
+  }
+}
+
+// d[row] = 1 - (k_row . ksum) / (|k_row| |ksum|); the cosine with the centroid equals the cosine
+// with the column sum.  A zero vector has cosine 0.  One warp per row, ksum staged in shared memory;
+// |ksum|^2 is folded by every warp in the same order, so all CTAs agree on it.
+template <int DT>
+__global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, int rows, int nvec,
+                                                   const float* __restrict__ ksum, float* __restrict__ d) {
+  constexpr int VEC = VecOf<DT>::n;
+  extern __shared__ float sh_ksum[];
+  const int C = nvec * VEC;
+  for (int c = threadIdx.x; c < C; c += blockDim.x) sh_ksum[c] = ksum[c];
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  float kn = 0.0f;
+  for (int v = lane; v < nvec; v += 32)
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) kn = __fmaf_rn(sh_ksum[v * VEC + e], sh_ksum[v * VEC + e], kn);
+  kn = warp_sum(kn);
+  const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
+  for (int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5); row < rows;
+       row += warps_total) {
+    const uint4* p = K + (size_t)row * nvec;
+    float dot = 0.0f, nrm = 0.0f;
+    for (int v0 = lane; v0 < nvec; v0 += 128) {
+      uint4 u[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (v0 + 32 * i < nvec) u[i] = ld_nc(p + v0 + 32 * i);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (v0 + 32 * i < nvec) {
+          float f[VEC];
+          unpack<DT>(u[i], f);
+          const float* ks = sh_ksum + (v0 + 32 * i) * VEC;
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) {
+            dot = __fmaf_rn(f[e], ks[e], dot);
+            nrm = __fmaf_rn(f[e], f[e], nrm);
+          }
+        }
+    }
+    dot = warp_sum(dot);
+    nrm = warp_sum(nrm);
+    if (lane == 0) {
+      float cosv = 0.0f;
+      if (nrm > 0.0f && kn > 0.0f) cosv = __fdiv_rn(dot, __fmul_rn(__fsqrt_rn(nrm), __fsqrt_rn(kn)));
+      d[row] = 1.0f - cosv;
+    }
+  }
+}
+
+}  // namespace ovggt

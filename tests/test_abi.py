@@ -1,0 +1,97 @@
+"""CPU checks of the C-ABI library: it loads, exports every symbol the header declares, and its
+host-side validation answers with the documented error codes before touching a GPU."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2603_05959_b200 import binding as B
+from paper_2603_05959_b200 import build as build_mod
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build_mod.build()
+    return B.lib()
+
+
+def declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(ovggt_\w+)\s*\(", text))
+    return names
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = declared_symbols()
+    assert len(names) >= 20
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in include/ but not exported"
+    assert set(B.EXPORTED) == names
+
+
+def _cfg(**over):
+    kw = dict(n_layers=1, n_heads=4, head_dim=64, n_special=5, grid_h=8, grid_w=8, budget=256,
+              anchor_tokens=8, k_max=3, min_anchor_interval=4, tau=0.2, alpha=0.5, beta=0.5,
+              protect_first_frame=1, score_mode=0, dtype=0)
+    kw.update(over)
+    budgets = (C.c_int32 * kw["n_layers"])(*([kw.pop("budget")] * kw["n_layers"]))
+    cfg = B.OvggtConfig(kw["n_layers"], kw["n_heads"], kw["head_dim"], kw["n_special"], kw["grid_h"],
+                        kw["grid_w"], budgets, kw["anchor_tokens"], kw["k_max"], kw["min_anchor_interval"],
+                        kw["tau"], kw["alpha"], kw["beta"], kw["protect_first_frame"], kw["score_mode"],
+                        kw["dtype"], None, 0)
+    cfg._keep = budgets
+    return cfg
+
+
+def test_workspace_bytes_is_a_pure_host_function(lib):
+    cfg = _cfg()
+    need = lib.ovggt_workspace_bytes(C.byref(cfg))
+    M, Cdim, R = 69, 256, 256 + 69
+    assert need >= 4 * R * Cdim * 4              # two K and two V buffers of B + M rows, fp32
+    big = lib.ovggt_workspace_bytes(C.byref(_cfg(budget=512)))
+    assert big > need
+    # the bf16 VGGT-shaped layer: 2 x 2 x (16384 + 1374) x 1024 x 2 bytes of K/V
+    need2 = lib.ovggt_workspace_bytes(C.byref(_cfg(n_heads=16, grid_h=37, grid_w=37, budget=16384,
+                                                    anchor_tokens=64, dtype=1)))
+    assert need2 >= 4 * 17758 * 1024 * 2 and need2 < 3 * 4 * 17758 * 1024 * 2
+
+
+def test_create_reports_config_errors_without_a_gpu(lib):
+    h = C.c_void_p()
+    bad = [(_cfg(head_dim=32), -1), (_cfg(n_layers=0, budget=256), -1), (_cfg(dtype=7), -1),
+           (_cfg(alpha=1.5), -1), (_cfg(k_max=17), -1), (_cfg(anchor_tokens=65), -1),
+           (_cfg(budget=68), -3), (_cfg(budget=69 + 3 * 8 - 1), -3)]
+    for cfg, code in bad:
+        assert lib.ovggt_workspace_bytes(C.byref(cfg)) == 0
+        assert lib.ovggt_cache_create(C.byref(cfg), C.byref(h)) == code
+        assert not h.value
+    ok = _cfg(budget=69 + 3 * 8)
+    assert lib.ovggt_workspace_bytes(C.byref(ok)) > 0
+    assert lib.ovggt_cache_create(C.byref(ok), C.byref(h)) == -1          # no workspace given
+    ok.workspace, ok.workspace_bytes = 1024 + 16, 1 << 40
+    assert lib.ovggt_cache_create(C.byref(ok), C.byref(h)) == -5          # misaligned workspace
+    ok.workspace, ok.workspace_bytes = 4096, 1024
+    assert lib.ovggt_cache_create(C.byref(ok), C.byref(h)) == -6          # workspace too small
+    assert lib.ovggt_cache_create(None, C.byref(h)) == -1
+    assert lib.ovggt_cache_destroy(None) == -1
+
+
+def test_null_handle_and_strerror(lib):
+    io = B.OvggtFrameIO()
+    for name in ("ovggt_layer_attend", "ovggt_layer_compress", "ovggt_layer_step", "ovggt_layer_step_host"):
+        assert getattr(lib, name)(None, 0, C.byref(io), None) == -1
+    st = B.OvggtStats()
+    assert lib.ovggt_cache_stats(None, 0, C.byref(st)) == -1
+    seen = {lib.ovggt_strerror(c) for c in range(0, -11, -1)}
+    assert len(seen) == 11 and b"unknown error" not in seen
+    assert lib.ovggt_strerror(-99) == b"unknown error"
+    assert lib.ovggt_kernel_launches() == 0
+    assert lib.ovggt_k_row_norms(None, 1, 64, 0, None, None) == -1
+    assert lib.ovggt_k_select(None, None, 0, 0, 1, None, None, None) == -1

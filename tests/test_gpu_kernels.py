@@ -1,0 +1,152 @@
+"""GPU parity of each kernel against the CPU oracle, through the C ABI (binding -> libovggt.so)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2603_05959_b200 import binding as B
+from paper_2603_05959_b200 import inputs as gen
+
+pytestmark = pytest.mark.gpu
+
+# Tolerances (derived from the arithmetic):
+#  fp32 fixed-order sums of <= 1024 squares against fp64: relative 1e-5
+#  d = 1 - cos with an fp32 column sum over up to ~32K rows: absolute 5e-6
+#  bf16 attention against the fp64 oracle: max-abs 2e-2, mean-abs 2e-3; fp32 attention: 1e-4
+NORM_RTOL = 1e-5
+DIV_ATOL = 5e-6
+ATT_MAX, ATT_MEAN, ATT_F32 = 2e-2, 2e-3, 1e-4
+
+
+def dev(x, dtype):
+    t = torch.from_numpy(np.ascontiguousarray(x))
+    return t.to(torch.bfloat16 if dtype == gen.DTYPE_BF16 else torch.float32).cuda()
+
+
+def rnd(shape, dtype, seed, scale=1.0):
+    x = np.random.default_rng(seed).standard_normal(shape).astype(np.float32) * np.float32(scale)
+    return gen.round_to_dtype(x, dtype)
+
+
+@pytest.mark.parametrize("rows,C,dtype", [(1374, 1024, 1), (69, 256, 0), (7, 64, 1), (1, 64, 0), (333, 768, 1),
+                                          (100, 1024, 0)])
+def test_row_norms(rows, C, dtype):
+    x = rnd((rows, C), dtype, 1) * np.exp(np.random.default_rng(2).normal(0, 0.75, (rows, 1))).astype(np.float32)
+    x = gen.round_to_dtype(x, dtype)
+    got = B.k_row_norms(dev(x, dtype)).cpu().numpy()
+    np.testing.assert_allclose(got, orc.residual_norms(x), rtol=NORM_RTOL)
+
+
+def test_row_norms_is_deterministic_and_handles_zero_rows():
+    x = dev(rnd((500, 1024), 1, 3), 1)
+    a, b = B.k_row_norms(x), B.k_row_norms(x)
+    assert torch.equal(a, b)
+    z = torch.zeros((4, 256), dtype=torch.float32, device="cuda")
+    assert torch.equal(B.k_row_norms(z), torch.zeros(4, device="cuda"))
+    assert B.k_row_norms(torch.empty((0, 256), dtype=torch.float32, device="cuda")).numel() == 0
+
+
+@pytest.mark.parametrize("rows,C,dtype", [(3000, 1024, 1), (325, 256, 0), (1, 64, 1), (17, 128, 0), (16384, 1024, 1)])
+def test_diversity(rows, C, dtype):
+    K = rnd((rows, C), dtype, 4) + np.float32(0.25)      # a non-zero centroid
+    K = gen.round_to_dtype(K, dtype)
+    got = B.k_diversity(dev(K, dtype)).cpu().numpy()
+    np.testing.assert_allclose(got, orc.diversity(K), rtol=0, atol=DIV_ATOL)
+
+
+def test_diversity_degenerate_rows():
+    K = np.zeros((5, 64), np.float32)
+    K[0, 0] = 1.0; K[1, 0] = 2.0; K[2, 0] = -1.0; K[4, 1] = 3.0
+    got = B.k_diversity(dev(K, 0)).cpu().numpy()
+    np.testing.assert_allclose(got, orc.diversity(K), atol=DIV_ATOL)
+    assert got[3] == 1.0                                  # a zero key: cosine 0 by convention
+
+
+def _select_case(N, seed, levels=None, specials=True, p_prot=0.1):
+    rng = np.random.default_rng(seed)
+    r = rng.random(N).astype(np.float32) if levels is None else \
+        (rng.integers(0, levels, N).astype(np.float32) / np.float32(levels))
+    if specials and N > 8:
+        r[rng.integers(0, N, 4)] = [np.nan, -np.inf, np.inf, -0.0]
+    flags = (rng.random(N) < p_prot).astype(np.uint8) * rng.integers(1, 3, N).astype(np.uint8)
+    return r, flags
+
+
+@pytest.mark.parametrize("N", [5, 325, 1500, 17758, 34142, 70001])
+@pytest.mark.parametrize("levels", [None, 3])
+def test_select_bit_exact(N, levels):
+    r, flags = _select_case(N, N + (levels or 0), levels)
+    P = int(np.count_nonzero(flags))
+    for Bud in sorted({P, P + 1, (P + N) // 2, N - 1, N, N + 5}):
+        got = B.k_select(torch.from_numpy(r).cuda(), torch.from_numpy(flags).cuda(), Bud).cpu().numpy()
+        np.testing.assert_array_equal(got, orc.select(r, flags, Bud))
+
+
+def test_select_batched_and_all_equal():
+    N, Bud, batch = 4000, 1500, 5
+    rs, fs = zip(*[_select_case(N, 50 + b, 4 if b % 2 else None) for b in range(batch)])
+    r = np.stack(rs); f = np.stack(fs)
+    r[4] = 0.25                                           # every priority equal: pure position order
+    got = B.k_select(torch.from_numpy(r).cuda(), torch.from_numpy(f).cuda(), Bud).cpu().numpy()
+    for b in range(batch):
+        np.testing.assert_array_equal(got[b], orc.select(r[b], f[b], Bud))
+
+
+@pytest.mark.parametrize("C,dtype", [(1024, 1), (256, 0), (64, 1)])
+def test_compact_is_exact_gather(C, dtype):
+    rng = np.random.default_rng(7)
+    N = 3001
+    k, v = rnd((N, C), dtype, 8), rnd((N, C), dtype, 9)
+    surv = np.sort(rng.choice(N, 1777, replace=False)).astype(np.int32)
+    kd, vd = B.k_compact(dev(k, dtype), dev(v, dtype), torch.from_numpy(surv).cuda())
+    assert np.array_equal(kd.float().cpu().numpy(), k[surv]) and np.array_equal(vd.float().cpu().numpy(), v[surv])
+    kd, vd = B.k_compact(dev(k, dtype), dev(v, dtype), torch.empty(0, dtype=torch.int32, device="cuda"))
+    assert kd.shape[0] == 0
+
+
+def _attn_check(M, N, H, dtype, seed, rows=None, qscale=1.0):
+    q, k, v = rnd((M, H * 64), dtype, seed, qscale), rnd((N, H * 64), dtype, seed + 1), rnd((N, H * 64), dtype, seed + 2)
+    got = B.k_attention(dev(q, dtype), dev(k, dtype), dev(v, dtype), H).float().cpu().numpy()
+    assert np.isfinite(got).all()
+    ref = orc.attention(q, k, v, H, 64, rows=rows)
+    g = got if rows is None else got[rows]
+    err = np.abs(g - ref)
+    if dtype == gen.DTYPE_F32:
+        assert err.max() <= ATT_F32
+    else:
+        assert err.max() <= ATT_MAX and err.mean() <= ATT_MEAN, (err.max(), err.mean())
+    return got
+
+
+@pytest.mark.parametrize("M,N,H", [(128, 128, 1), (1, 1, 1), (94, 129, 2), (200, 1000, 2), (69, 325, 4),
+                                   (300, 4096, 3), (129, 2500, 1)])
+def test_attention_bf16_small(M, N, H):
+    orc.set_threads(8)
+    _attn_check(M, N, H, gen.DTYPE_BF16, 10 + M + N)
+
+
+def test_attention_bf16_large_logits_exercise_rescaling():
+    orc.set_threads(8)
+    _attn_check(150, 1500, 2, gen.DTYPE_BF16, 77, qscale=6.0)
+
+
+@pytest.mark.parametrize("M,N,H", [(69, 325, 4), (1, 1, 1), (130, 700, 2)])
+def test_attention_fp32(M, N, H):
+    orc.set_threads(8)
+    _attn_check(M, N, H, gen.DTYPE_F32, 20 + M)
+
+
+def test_attention_bf16_full_size_sampled_rows():
+    """The bench configuration: 1374 queries x 17758 keys x 16 heads; the oracle checks sampled rows."""
+    orc.set_threads(max(1, min(32, torch.get_num_threads())))
+    rows = np.sort(np.random.default_rng(5).choice(1374, 24, replace=False)).astype(np.int32)
+    rows[0], rows[-1] = 0, 1373
+    got = _attn_check(1374, 17758, 16, gen.DTYPE_BF16, 30, rows=rows)
+    # properties that hold at any size: finite, and each output inside the range of V per column
+    assert np.abs(got).max() < 6.0
+
+
+def test_attention_is_deterministic():
+    q, k, v = (dev(rnd(s, 1, i), 1) for i, s in enumerate(((500, 256), (3000, 256), (3000, 256))))
+    a, b = B.k_attention(q, k, v, 4), B.k_attention(q, k, v, 4)
+    assert torch.equal(a, b)
