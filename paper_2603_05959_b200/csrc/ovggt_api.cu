@@ -649,6 +649,7 @@ extern "C" const char* ovggt_strerror(int code) {
 // ------------------------------------------------------------------ single kernels
 
 extern "C" int ovggt_k_row_norms(const void* x, int32_t rows, int32_t C, int32_t dtype, float* s, void* stream) {
+  if (rows == 0) return OVGGT_OK;
   if (!x || !s || rows < 0 || C < 1 || (C * elem_bytes(dtype)) % 16 || (dtype != kF32 && dtype != kBF16))
     return OVGGT_ERR_INVALID_ARG;
   if (!aligned16(x)) return OVGGT_ERR_MISALIGNED;
@@ -662,6 +663,7 @@ extern "C" size_t ovggt_k_diversity_scratch_bytes(int32_t rows, int32_t C) {
 
 extern "C" int ovggt_k_diversity(const void* K, int32_t rows, int32_t C, int32_t dtype, float* d, void* scratch,
                                  void* stream) {
+  if (rows == 0) return OVGGT_OK;
   if (!K || !d || !scratch || rows < 0 || C < 1 || (C * elem_bytes(dtype)) % 16 || (dtype != kF32 && dtype != kBF16) ||
       (size_t)C * 4 > 48 * 1024)
     return OVGGT_ERR_INVALID_ARG;
@@ -673,7 +675,9 @@ extern "C" int ovggt_k_diversity(const void* K, int32_t rows, int32_t C, int32_t
 
 extern "C" int ovggt_k_select(const float* r, const uint8_t* flags, int32_t N, int32_t B, int32_t batch,
                               int32_t* survivors, void* scratch, void* stream) {
-  if (!r || !flags || !survivors || !scratch || N < 1 || B < 0 || batch < 1) return OVGGT_ERR_INVALID_ARG;
+  if (N < 1 || B < 0 || batch < 1) return OVGGT_ERR_INVALID_ARG;
+  if (B == 0) return OVGGT_OK;   // nothing can be kept: the survivor lists are empty
+  if (!r || !flags || !survivors || !scratch) return OVGGT_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int* status = reinterpret_cast<int*>(scratch);
   uint32_t* gkeys = reinterpret_cast<uint32_t*>(static_cast<char*>(scratch) + 64);
@@ -694,6 +698,7 @@ extern "C" int ovggt_k_select(const float* r, const uint8_t* flags, int32_t N, i
 
 extern "C" int ovggt_k_compact(const void* k_src, const void* v_src, const int32_t* survivors, int32_t n_keep,
                                int32_t C, int32_t dtype, void* k_dst, void* v_dst, void* stream) {
+  if (n_keep == 0) return OVGGT_OK;
   if (!k_src || !v_src || !survivors || !k_dst || !v_dst || n_keep < 0 || C < 1 || (C * elem_bytes(dtype)) % 16)
     return OVGGT_ERR_INVALID_ARG;
   if (!aligned16(k_src) || !aligned16(v_src) || !aligned16(k_dst) || !aligned16(v_dst)) return OVGGT_ERR_MISALIGNED;
