@@ -53,7 +53,8 @@ enum {
   OVGGT_ERR_CUDA = -7,              /* a CUDA runtime / driver call failed; see ovggt_last_cuda_error */
   OVGGT_ERR_DEVICE_STATUS = -8,     /* a kernel reported an inconsistency through the device status word */
   OVGGT_ERR_TIMEOUT = -9,           /* a bounded device-side wait ran out (the kernel returned cleanly) */
-  OVGGT_ERR_UNSUPPORTED = -10       /* the configuration is valid but this build has no kernel for it */
+  OVGGT_ERR_UNSUPPORTED = -10,      /* the configuration is valid but this build has no kernel for it */
+  OVGGT_ERR_TOO_LARGE = -11         /* a size exceeds the fixed capacity of a built-in scratch array */
 };
 
 enum { OVGGT_DTYPE_F32 = 0, OVGGT_DTYPE_BF16 = 1 };
@@ -193,6 +194,23 @@ int ovggt_k_row_norms(const void* x, int32_t rows, int32_t C, int32_t dtype, flo
 size_t ovggt_k_diversity_scratch_bytes(int32_t rows, int32_t C);
 int ovggt_k_diversity(const void* K, int32_t rows, int32_t C, int32_t dtype, float* d, void* scratch,
                       void* stream);
+
+/* (No counterpart in the paper: a packaging variant of ovggt_k_diversity.)
+ * The same result, d[i] = 1 - cos(K[i, :], sum of all rows of K), for callers that must not allocate device
+ * memory and have no spare buffer to lend: code that runs after its host application has handed the whole GPU
+ * to a pool allocator, inside a latency-bound frame loop where a driver allocation would stall the device, or
+ * behind a plug-in interface that forbids allocation calls.  The intermediate column sums live in an array that
+ * is compiled into the library (about 2.4 MB on every GPU that loads it, held until the process exits), so the
+ * call needs K and d only and itself calls no allocating routine of CUDA or of any other library.
+ *   Limit: C <= 1024 columns (any number of rows); a larger C returns OVGGT_ERR_TOO_LARGE and launches nothing.
+ *   The first call on each device looks the array's device address up (cudaGetSymbolAddress, with that device
+ *   current) before it launches; make that first call outside any stream capture.  Later calls on the device
+ *   only launch kernels.
+ *   All calls on a device share the one array, and it keeps whatever the previous call left in it.  Nothing in
+ *   it has to start at zero: each call overwrites every element it later reads.  Two calls that overlap on the
+ *   GPU (different streams, or different host threads without ordering) race on it; order them on one stream
+ *   or with events. */
+int ovggt_k_diversity_static(const void* K, int32_t rows, int32_t C, int32_t dtype, float* d, void* stream);
 
 /* Eq. 8: survivors of N candidates with priorities r [N] and flags [N] (non-zero = protected) under budget B:
  * every protected row plus the B - |P| evictable rows of largest r, ties to the lower position, NaN ranks

@@ -27,7 +27,7 @@ EXPORTED = [
     "ovggt_cache_export", "ovggt_cache_import", "ovggt_cache_last_selection", "ovggt_kernel_launches",
     "ovggt_cache_profile_enable", "ovggt_cache_profile_read",
     "ovggt_strerror", "ovggt_last_cuda_error", "ovggt_k_row_norms", "ovggt_k_diversity_scratch_bytes",
-    "ovggt_k_diversity", "ovggt_k_select", "ovggt_k_compact", "ovggt_k_attention_scratch_bytes",
+    "ovggt_k_diversity", "ovggt_k_diversity_static", "ovggt_k_select", "ovggt_k_compact", "ovggt_k_attention_scratch_bytes",
     "ovggt_k_attention",
 ]
 
@@ -101,6 +101,7 @@ def lib():
         L.ovggt_k_diversity_scratch_bytes.restype = C.c_size_t
         L.ovggt_k_diversity_scratch_bytes.argtypes = [i32, i32]
         L.ovggt_k_diversity.argtypes = [vp, i32, i32, i32, vp, vp, vp]
+        L.ovggt_k_diversity_static.argtypes = [vp, i32, i32, i32, vp, vp]
         L.ovggt_k_select.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
         L.ovggt_k_compact.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp]
         L.ovggt_k_attention_scratch_bytes.restype = C.c_size_t
@@ -294,6 +295,15 @@ def k_diversity(K: torch.Tensor, stream=None) -> torch.Tensor:
                           device=K.device)
     _check(lib().ovggt_k_diversity(_dptr(K), K.shape[0], K.shape[1], dtype, _dptr(d), _dptr(scratch),
                                    _stream_ptr(stream)), "ovggt_k_diversity")
+    return d
+
+
+def k_diversity_static(K: torch.Tensor, d: torch.Tensor, stream=None) -> torch.Tensor:
+    """ovggt_k_diversity_static: the caller passes the input K and the output d only; the scratch is an array
+    built into the library, so the call allocates nothing (d is given, not created here)."""
+    dtype = DTYPE_F32 if K.dtype == torch.float32 else DTYPE_BF16
+    _check(lib().ovggt_k_diversity_static(_dptr(K), K.shape[0], K.shape[1], dtype, _dptr(d), _stream_ptr(stream)),
+           "ovggt_k_diversity_static")
     return d
 
 

@@ -642,6 +642,7 @@ extern "C" const char* ovggt_strerror(int code) {
     case OVGGT_ERR_DEVICE_STATUS: return "a kernel reported an inconsistency";
     case OVGGT_ERR_TIMEOUT: return "a bounded device-side wait ran out";
     case OVGGT_ERR_UNSUPPORTED: return "configuration not supported by this build";
+    case OVGGT_ERR_TOO_LARGE: return "size exceeds the fixed capacity of the built-in scratch array";
     default: return "unknown error";
   }
 }
@@ -716,4 +717,48 @@ extern "C" int ovggt_k_attention(const void* q, const void* k, const void* v, in
   if (dtype == kBF16 && (!scratch || !device_status)) return OVGGT_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return OVGGT_ERR_MISALIGNED;
   return launch_attention(q, k, v, M, N, n_heads, dtype, out, scratch, device_status, static_cast<cudaStream_t>(stream));
+}
+
+// ------------------------------------------------------------------ allocation-free diversity
+
+namespace {
+constexpr int kStaticDivMaxC = 1024;
+// Built-in scratch of ovggt_k_diversity_static: column-sum partials [kMaxColsumParts, C] followed by the column
+// sums [C], C <= kStaticDivMaxC (about 2.4 MB).  Every GPU that loads the library holds it until the process exits.
+static __device__ __align__(256) float g_static_div_scratch[(kMaxColsumParts + 1) * kStaticDivMaxC];
+
+constexpr int kMaxDevices = 64;
+float* g_static_div_ptr[kMaxDevices] = {nullptr};
+std::atomic<int> g_static_div_ready[kMaxDevices];
+
+// Device address of the built-in scratch on the current device.  In host code the array's name is only a
+// handle for the runtime, not an address a kernel could use; the address is asked for once per device.
+int static_div_scratch(float** out) {
+  int dev = 0;
+  CK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return OVGGT_ERR_UNSUPPORTED;
+  if (!g_static_div_ready[dev].load(std::memory_order_acquire)) {
+    void* p = nullptr;
+    CK(cudaGetSymbolAddress(&p, g_static_div_scratch));
+    g_static_div_ptr[dev] = static_cast<float*>(p);
+    g_static_div_ready[dev].store(1, std::memory_order_release);
+  }
+  *out = g_static_div_ptr[dev];
+  return OVGGT_OK;
+}
+}  // namespace
+
+extern "C" int ovggt_k_diversity_static(const void* K, int32_t rows, int32_t C, int32_t dtype, float* d,
+                                        void* stream) {
+  if (rows == 0) return OVGGT_OK;
+  if (!K || !d || rows < 0 || C < 1 || (dtype != kF32 && dtype != kBF16) || (C * elem_bytes(dtype)) % 16)
+    return OVGGT_ERR_INVALID_ARG;
+  if (C > kStaticDivMaxC) return OVGGT_ERR_TOO_LARGE;
+  if (!aligned16(K)) return OVGGT_ERR_MISALIGNED;
+  float* scratch = nullptr;
+  int rc = static_div_scratch(&scratch);
+  if (rc) return rc;
+  float* part = scratch;
+  float* ksum = scratch + (size_t)kMaxColsumParts * C;
+  return launch_diversity(K, rows, C, dtype, part, ksum, d, static_cast<cudaStream_t>(stream));
 }
