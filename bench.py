@@ -312,7 +312,7 @@ def run_ours(args) -> None:
         N = Bud + M
         attn_flops = 4.0 * M * N * C
         attn_ms = prof["attention"]["ms"] / max(1, prof["attention"]["count"])
-        achieved = attn_flops / (attn_ms * 1e-3) / 1e12
+        achieved = attn_flops / (attn_ms * 1e-3) / 1e12 if attn_ms > 0 else 0.0
         peak = float(peaks["bf16_tflops"])
         eb = cfg.elem_bytes
         kernels = {}

@@ -214,8 +214,9 @@ int ovggt_k_diversity_static(const void* K, int32_t rows, int32_t C, int32_t dty
 
 /* Eq. 8: survivors of N candidates with priorities r [N] and flags [N] (non-zero = protected) under budget B:
  * every protected row plus the B - |P| evictable rows of largest r, ties to the lower position, NaN ranks
- * with -inf.  survivors [min(N, B)] ascending.  scratch: device, >= 4 * N + 64 bytes.
- * `batch` independent problems are laid out back to back (r, flags, survivors strides N, N, B); one CTA each. */
+ * with -inf.  survivors [min(N, B)] ascending.  scratch: device, >= 64 bytes (a status word).
+ * `batch` independent problems are laid out back to back (r, flags, survivors strides N, N, min(N, B)); one
+ * thread-block cluster each.  N up to about 350,000 (8 CTAs x shared memory); beyond: OVGGT_ERR_UNSUPPORTED. */
 int ovggt_k_select(const float* r, const uint8_t* flags, int32_t N, int32_t B, int32_t batch,
                    int32_t* survivors, void* scratch, void* stream);
 

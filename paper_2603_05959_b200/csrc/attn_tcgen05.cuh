@@ -1,12 +1,13 @@
 // bf16 flash attention for sm_100a: out = softmax(Q K^T / sqrt(64)) V per head, head_dim 64, no mask.
 //
 // One CTA owns one 128-row query tile of one head and a contiguous range of 128-row KV tiles.
-//   warp 0      TMA producer: Q once, then K and V tiles into 128-byte-swizzled shared-memory stages
-//   warp 1      allocates tensor memory and issues tcgen05.mma:  S = Q K^T  (SS, fp32 in TMEM),
-//               O += P V (P read from TMEM as the A operand, V MN-major from shared memory)
-//   warps 2-5   softmax: one thread per query row reads its S row with tcgen05.ld, keeps a running
+//   warps 0-3   softmax: one thread per query row reads its S row with tcgen05.ld, keeps a running
 //               reference maximum (rescaling O only when the maximum grows by more than 2^8), writes
 //               P as bf16 over the S columns, and at the end normalises and stores O
+//   warp 4      TMA producer: Q once, then K and V tiles into 128-byte-swizzled shared-memory stages
+//   warp 5      allocates tensor memory and issues tcgen05.mma:  S = Q K^T  (SS, fp32 in TMEM),
+//               O += P V (P read from TMEM as the A operand, V MN-major from shared memory)
+//   warps 6-7   only complete the second warpgroup, which hands its registers to the softmax warpgroup
 // Two CTAs are resident per SM (256 TMEM columns and ~82 KB shared memory each), so one CTA's MMAs
 // overlap the other's exponentials.  The KV range may be split across CTAs; partial (O, max, sum)
 // triples are merged by a second kernel.  Every mbarrier wait is bounded: on expiry the CTA records
@@ -23,7 +24,8 @@ constexpr int kBM = 128;            // query rows per CTA
 constexpr int kBN = 128;            // KV rows per tile
 constexpr int kHD = 64;             // head dim
 constexpr int kKVStages = 2;
-constexpr int kAttnThreads = 192;
+constexpr int kAttnThreads = 256;
+constexpr int kRegsSoftmax = 216, kRegsOther = 40;   // 2 CTAs x (128 x 216 + 128 x 40) = 64K registers
 constexpr int kTileBytes = kBN * kHD * 2;          // 16 KB
 constexpr int kTmemCols = 256;
 constexpr int kColS = 0, kColO = 128;
@@ -162,6 +164,28 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// (a.x * b.x + c.x, a.y * b.y + c.y) and (a.x + b.x, a.y + b.y) as single packed instructions
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("{\n .reg .b64 ra, rb, rc, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rb, {%4, %5};\n mov.b64 rc, {%6, %7};\n"
+      " fma.rn.f32x2 rd, ra, rb, rc;\n mov.b64 {%0, %1}, rd;\n}\n"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+  return d;
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+  float2 d;
+  asm("{\n .reg .b64 ra, rb, rd;\n mov.b64 ra, {%2, %3};\n mov.b64 rb, {%4, %5};\n"
+      " add.rn.f32x2 rd, ra, rb;\n mov.b64 {%0, %1}, rd;\n}\n"
+      : "=f"(d.x), "=f"(d.y)
+      : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t d;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
@@ -211,7 +235,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {
+  if (warp == 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&B->tmem_base)),
                  "r"((uint32_t)kTmemCols)
                  : "memory");
@@ -222,7 +246,9 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem = *(volatile uint32_t*)&B->tmem_base;
 
-  if (warp == 0) {
+  if (warp >= 4) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+  if (warp == 4) {
     // ------------------------------------------------ TMA producer
     if (lane == 0) {
       int issued_k = 0, issued_v = 0;
@@ -254,7 +280,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
+  } else if (warp == 5) {
     // ------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc_qk = idesc_bf16(kBN, false);
@@ -293,9 +319,11 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
     }
     __syncwarp();
+  }
   } else {
     // ------------------------------------------------ softmax, correction and epilogue (128 threads)
-    const int quad = warp & 3;
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+    const int quad = warp;
     const int row = quad * 32 + lane;
     const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16);
     const float c = 1.4426950408889634f * 0.125f;     // log2(e) / sqrt(64)
@@ -315,10 +343,16 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         for (int j = 0; j < 128; ++j)
           if (col0 + j >= P.N) s[j] = 0xFF800000u;     // -inf on columns past the last row
       }
-      float mx = __uint_as_float(s[0]);
+      // row maximum: four independent chains of 3-input maxima
+      float m4[4];
 #pragma unroll
-      for (int j = 1; j < 128; ++j) mx = fmaxf(mx, __uint_as_float(s[j]));
-      mx *= c;
+      for (int q = 0; q < 4; ++q) {
+        m4[q] = fmaxf(__uint_as_float(s[32 * q]), __uint_as_float(s[32 * q + 1]));
+#pragma unroll
+        for (int j = 2; j < 32; j += 2)
+          m4[q] = max3(m4[q], __uint_as_float(s[32 * q + j]), __uint_as_float(s[32 * q + j + 1]));
+      }
+      float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * c;
       if (it == 0) {
         mref = mx;
       } else {
@@ -340,17 +374,20 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
         }
       }
-      const float nm = -mref;
-      float sum = 0.0f;
+      // p = 2^(s * c - mref) on pairs; four independent packed partial sums, folded in a fixed order
+      const float2 c2 = make_float2(c, c), nm2 = make_float2(-mref, -mref);
+      float2 acc[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) acc[q] = make_float2(0.0f, 0.0f);
 #pragma unroll
       for (int j = 0; j < 128; j += 2) {
-        const float p0 = ex2(fmaf(__uint_as_float(s[j]), c, nm));
-        const float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), c, nm));
-        sum += p0;
-        sum += p1;
-        s[j >> 1] = pack_bf16(p0, p1);
+        const float2 x = fma2(make_float2(__uint_as_float(s[j]), __uint_as_float(s[j + 1])), c2, nm2);
+        const float2 p = make_float2(ex2(x.x), ex2(x.y));
+        acc[(j >> 1) & 3] = add2(acc[(j >> 1) & 3], p);
+        s[j >> 1] = pack_bf16(p.x, p.y);
       }
-      l += sum;
+      const float2 t = add2(add2(acc[0], acc[1]), add2(acc[2], acc[3]));
+      l += t.x + t.y;
       tmem_st32(t_row + kColS, s);
       tmem_st32(t_row + kColS + 32, s + 32);
       tmem_wait_st();
@@ -393,7 +430,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   // ------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == 5) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols) : "memory");
   }

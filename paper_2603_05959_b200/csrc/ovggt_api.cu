@@ -50,10 +50,24 @@ constexpr size_t kSmemLimit = 227 * 1024;
 
 int colsum_parts(int rows) { return std::max(1, std::min(kMaxColsumParts, (rows + 15) / 16)); }
 
-size_t select_smem_bytes(int N, int M, bool keys_in_smem) {
-  size_t b = align_up(sizeof(SelectShared), 16) + align_up((size_t)M * 4, 16) + (size_t)N;
-  if (keys_in_smem) b += (size_t)N * 4;
-  return b + 16;
+// CTAs per cluster of the selection kernels: about 2K candidates per CTA, at most 8 (the portable limit).
+int select_cluster_ctas(int N) { return std::max(1, std::min(kSelectMaxCtas, (N + 2047) / 2048)); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_cluster(void (*kernel)(KArgs...), dim3 grid, int ncta, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kSelectThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = ncta;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 // ------------------------------------------------------------------ single-kernel launchers
@@ -133,7 +147,6 @@ struct LayerState {
   float* stored[2];
   float *s_raw, *d, *r;
   int* surv;
-  uint32_t* gkeys;
   int* n_keep_dev;
   size_t kv_bytes = 0;
 };
@@ -244,7 +257,6 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
     off[i++] = L.take(R * 4);           // d
     off[i++] = L.take(R * 4);           // r
     off[i++] = L.take(R * 4);           // survivors
-    off[i++] = L.take(R * 4);           // gkeys
     off[i++] = L.take(64);              // n_keep
     if (h) {
       LayerState& S = h->layers[l];
@@ -258,7 +270,6 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
       S.d = reinterpret_cast<float*>(base + off[i++]);
       S.r = reinterpret_cast<float*>(base + off[i++]);
       S.surv = reinterpret_cast<int*>(base + off[i++]);
-      S.gkeys = reinterpret_cast<uint32_t*>(base + off[i++]);
       S.n_keep_dev = reinterpret_cast<int*>(base + off[i++]);
       S.budget = c->budget[l];
       S.kv_bytes = 4 * R * C * eb;
@@ -435,19 +446,15 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
   P.s_raw = S.s_raw; P.d = S.d; P.conf = io->conf; P.override_r = io->score_override;
   P.ids_src = S.ids[b]; P.flags_src = S.flags[b]; P.stored_src = S.stored[b];
   P.ids_dst = S.ids[b ^ 1]; P.flags_dst = S.flags[b ^ 1]; P.stored_dst = S.stored[b ^ 1];
-  P.r_out = S.r; P.survivors = S.surv; P.gkeys = S.gkeys;
+  P.r_out = S.r; P.survivors = S.surv;
   P.status = h->status; P.n_keep_out = S.n_keep_dev;
-  size_t smem = select_smem_bytes(N, M, true);
-  P.keys_in_smem = 1;
-  if (smem > kSmemLimit) {
-    P.keys_in_smem = 0;
-    smem = select_smem_bytes(N, M, false);
-    if (smem > kSmemLimit) return OVGGT_ERR_UNSUPPORTED;
-  }
+  const int ncta = select_cluster_ctas(N);
+  const size_t smem = select_smem_bytes((N + ncta - 1) / ncta, h->Np);
+  if (smem > kSmemLimit) return OVGGT_ERR_UNSUPPORTED;
   CK(cudaFuncSetAttribute(k_compress_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit));
   {
     ProfScope ps(h, OVGGT_PROF_SELECT, st);
-    k_compress_select<<<1, kSelectThreads, smem, st>>>(P);
+    CK(launch_cluster(k_compress_select, dim3(ncta), ncta, smem, st, P));
     LAUNCHED();
   }
   const int n_keep = std::min(N, B);
@@ -681,18 +688,12 @@ extern "C" int ovggt_k_select(const float* r, const uint8_t* flags, int32_t N, i
   if (!r || !flags || !survivors || !scratch) return OVGGT_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int* status = reinterpret_cast<int*>(scratch);
-  uint32_t* gkeys = reinterpret_cast<uint32_t*>(static_cast<char*>(scratch) + 64);
-  size_t smem = align_up(sizeof(SelectShared), 16) + (size_t)N * 5 + 16;
-  int in_smem = 1;
-  if (smem > kSmemLimit || batch > 1) {
-    // batched problems keep their keys in global memory so that several CTAs fit on one SM
-    in_smem = smem <= 48 * 1024 ? 1 : 0;
-    if (!in_smem) smem = align_up(sizeof(SelectShared), 16) + (size_t)N + 16;
-    if (smem > kSmemLimit) return OVGGT_ERR_UNSUPPORTED;
-  }
+  const int ncta = select_cluster_ctas(N);
+  const size_t smem = select_smem_bytes((N + ncta - 1) / ncta, 0);
+  if (smem > kSmemLimit) return OVGGT_ERR_UNSUPPORTED;
   CK(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit));
   CK(cudaMemsetAsync(status, 0, 4, st));
-  k_select<<<batch, kSelectThreads, smem, st>>>(r, flags, N, B, survivors, gkeys, in_smem, status);
+  CK(launch_cluster(k_select, dim3(ncta, batch), ncta, smem, st, r, flags, (int)N, (int)B, (int*)survivors, status));
   LAUNCHED();
   return OVGGT_OK;
 }

@@ -1,80 +1,188 @@
-// Budgeted selection (Eq. 8) as a single-CTA radix select, and the fused per-step kernel that
-// prepares its input: anchor flags (Sec. 3.3), activation smoothing (Eq. 6), hybrid priorities (Eq. 7).
+// Budgeted selection (Eq. 8) as a radix select over a thread-block cluster, and the fused per-step kernel
+// that prepares its input: anchor flags (Sec. 3.3), activation smoothing (Eq. 6), hybrid priorities (Eq. 7).
 //
-// One CTA of 1024 threads holds all N keys and flags in shared memory (N <= ~44K; larger N keeps the
-// keys in a global scratch array).  The k-th largest key is found with four 8-bit most-significant-digit
-// passes; rows tied with it are admitted in position order, so the result is unique.
+// A cluster of up to 8 CTAs x 1024 threads splits the N candidates into contiguous position ranges, one per
+// CTA, held in that CTA's shared memory.  Protected rows get the largest possible key, so "every protected
+// row plus the B - |P| best evictable rows" is simply "the B largest keys"; ties at the threshold are
+// admitted in position order, so the result is unique.  The B-th largest key is found with four 8-bit
+// most-significant-digit passes; per-CTA digit histograms and counts are combined through distributed
+// shared memory with one cluster barrier per pass.
 #pragma once
+
+#include <cooperative_groups.h>
 
 #include "common.cuh"
 
 namespace ovggt {
 
+namespace cg = cooperative_groups;
+
 constexpr int kSelectThreads = 1024;
-constexpr uint8_t kKeepBit = 0x80;
+constexpr int kSelectMaxCtas = 8;
+constexpr uint32_t kKeyProtected = 0xFFFFFFFFu;   // above the key of +inf (0xFF800000)
 
 struct SelectShared {
-  int hist[256];
+  int hist[2][256];          // this CTA's digit histogram, double-buffered across passes (read by the cluster)
+  int tot[256];              // cluster-wide digit counts of the current pass
   int scan[64];
   float fscan[64];
   int digit, krem;
+  int pub_eq, pub_keep;      // this CTA's totals, read by the other CTAs of the cluster
+  float pub_lo_h, pub_hi_h, pub_lo_n, pub_hi_n;
 };
 
-// Selection core.  keys[N]: rank keys; flags[N]: low bits non-zero = protected (flags == nullptr: none);
-// bit 7 of flags is used as the keep mark when flags != nullptr, otherwise `mark` (N bytes) is used.
-// Writes survivors[0 .. n_keep) ascending and returns n_keep (= min(N, B) unless |P| > B, which sets *bad).
-__device__ inline int select_core(const uint32_t* keys, uint8_t* flags, uint8_t* mark, int N, int B,
-                                  int* survivors, SelectShared* sh, int* bad) {
-  const int tid = threadIdx.x, nthr = blockDim.x;
-  uint8_t* fl = flags ? flags : mark;
-  if (!flags)
-    for (int i = tid; i < N; i += nthr) mark[i] = 0;
-  __syncthreads();
-  int prot = 0;
-  for (int i = tid; i < N; i += nthr) prot += (fl[i] & 3) != 0;
-  prot = block_sum_int(prot, sh->scan);
-  const bool keep_all = N <= B;
-  int k = B - prot;
-  if (!keep_all && k < 0) {
-    if (tid == 0) *bad = 1;
-    k = 0;
+// Range of positions owned by CTA `rank` when N positions are split over `ncta` CTAs.
+__device__ __forceinline__ void cta_range(int N, int ncta, int rank, int* begin, int* end) {
+  const int span = (N + ncta - 1) / ncta;
+  *begin = min(N, rank * span);
+  *end = min(N, *begin + span);
+}
+
+// Warp 0 finds the digit whose bin holds the krem-th largest remaining key, given bin counts tot[256].
+__device__ __forceinline__ void find_digit(const int* tot, int krem, SelectShared* sh) {
+  const int tid = threadIdx.x;
+  if (tid < 32) {
+    int c[8], local = 0;
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+      c[b] = tot[tid * 8 + b];
+      local += c[b];
+    }
+    int above = local;   // inclusive suffix sum over lanes: keys in this lane's bins and in all higher bins
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int y = __shfl_down_sync(0xFFFFFFFFu, above, o);
+      if (tid + o < 32) above += y;
+    }
+    int cum = above - local;
+#pragma unroll
+    for (int b = 7; b >= 0; --b) {
+      if (cum < krem && cum + c[b] >= krem) {
+        sh->digit = tid * 8 + b;
+        sh->krem = krem - cum;
+      }
+      cum += c[b];
+    }
   }
+}
+
+// Digit histogram of the keys that match (mask, prefix).  Keys of one step share their leading bits, so lanes
+// of a warp mostly hit the same bin: lanes with equal digits are grouped and one of them adds the group's count.
+__device__ __forceinline__ void digit_histogram(const uint32_t* keys, int cnt, uint32_t mask, uint32_t prefix,
+                                                int shift, int* hist) {
+  const int tid = threadIdx.x, nthr = blockDim.x;
+  for (int i0 = 0; i0 < cnt; i0 += nthr) {
+    const int i = i0 + tid;
+    int digit = -1;
+    if (i < cnt) {
+      const uint32_t key = keys[i];
+      if ((key & mask) == prefix) digit = (int)((key >> shift) & 255u);
+    }
+    const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
+    if (digit >= 0 && (int)(__ffs(peers) - 1) == (tid & 31)) atomicAdd(&hist[digit], __popc(peers));
+  }
+}
+
+// keys[0 .. cnt): this CTA's keys for positions [begin, begin + cnt).  Finds the B largest keys of the whole
+// cluster (ties by position), writes the surviving global positions, ascending, to survivors[] and marks the
+// kept local positions in keep[] (cnt bytes).  Returns the cluster-wide survivor count, min(N, B).
+// *my_base receives the index in survivors[] of this CTA's first survivor.
+__device__ inline int cluster_select(cg::cluster_group& cluster, const uint32_t* keys, uint8_t* keep, int begin,
+                                     int cnt, int N, int B, int* survivors, SelectShared* sh, int* my_base,
+                                     int* bad) {
+  const int tid = threadIdx.x, nthr = blockDim.x;
+  const int ncta = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+  const bool keep_all = N <= B;
   uint32_t T = 0;
   int need_eq = 0;
-  if (!keep_all && k > 0) {
+  if (!keep_all) {
     uint32_t prefix = 0, mask = 0;
-    int krem = k;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-      for (int b = tid; b < 256; b += nthr) sh->hist[b] = 0;
+    int krem = B;
+    int buf = 0;
+    for (int shift = 24; shift >= 0; shift -= 8, buf ^= 1) {
+      int* hist = sh->hist[buf];
+      for (int b = tid; b < 256; b += nthr) hist[b] = 0;
       __syncthreads();
-      for (int i = tid; i < N; i += nthr)
-        if ((fl[i] & 3) == 0 && (keys[i] & mask) == prefix) atomicAdd(&sh->hist[(keys[i] >> shift) & 255], 1);
-      __syncthreads();
-      if (tid < 32) {
-        int c[8], local = 0;
-#pragma unroll
-        for (int b = 0; b < 8; ++b) {
-          c[b] = sh->hist[tid * 8 + b];
-          local += c[b];
-        }
-        // number of matching rows in bins above this lane's bins
-        int above = local;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          int y = __shfl_down_sync(0xFFFFFFFFu, above, o);
-          if (tid + o < 32) above += y;
-        }
-        above -= local;
-        int cum = above;
-#pragma unroll
-        for (int b = 7; b >= 0; --b) {
-          if (cum < krem && cum + c[b] >= krem) {
-            sh->digit = tid * 8 + b;
-            sh->krem = krem - cum;
-          }
-          cum += c[b];
-        }
+      digit_histogram(keys, cnt, mask, prefix, shift, hist);
+      cluster.sync();
+      // every CTA folds all histograms and finds the same digit
+      if (tid < 256) {
+        int t = 0;
+        for (int r = 0; r < ncta; ++r) t += cluster.map_shared_rank(hist, r)[tid];
+        sh->tot[tid] = t;
       }
+      __syncthreads();
+      find_digit(sh->tot, krem, sh);
+      __syncthreads();
+      prefix |= (uint32_t)sh->digit << shift;
+      mask |= 255u << shift;
+      krem = sh->krem;
+    }
+    T = prefix;
+    need_eq = krem;
+  }
+  // Thread t owns the contiguous local positions [t*chunk, (t+1)*chunk).
+  const int chunk = (cnt + nthr - 1) / nthr;
+  const int lo = min(cnt, tid * chunk), hi = min(cnt, lo + chunk);
+  int cnt_eq = 0;
+  if (!keep_all)
+    for (int i = lo; i < hi; ++i) cnt_eq += keys[i] == T;
+  int eq_total;
+  int eq_rank = block_excl_scan_int(cnt_eq, sh->scan, &eq_total);
+  if (tid == 0) sh->pub_eq = eq_total;
+  cluster.sync();
+  int eq_all = 0;
+  for (int r = 0; r < ncta; ++r) {
+    const int v = *cluster.map_shared_rank(&sh->pub_eq, r);
+    if (r < rank) eq_rank += v;
+    eq_all += v;
+  }
+  // more protected rows than the budget holds: only the first B of them can stay
+  *bad = (!keep_all && T == kKeyProtected && eq_all > need_eq) ? 1 : 0;
+  int cnt_keep = 0;
+  for (int i = lo; i < hi; ++i) {
+    bool k = true;
+    if (!keep_all) {
+      const uint32_t key = keys[i];
+      k = key > T || (key == T && eq_rank++ < need_eq);
+    }
+    keep[i] = k ? 1 : 0;
+    cnt_keep += k;
+  }
+  int keep_total;
+  int base = block_excl_scan_int(cnt_keep, sh->scan, &keep_total);
+  if (tid == 0) sh->pub_keep = keep_total;
+  cluster.sync();
+  int before = 0, all = 0;
+  for (int r = 0; r < ncta; ++r) {
+    const int v = *cluster.map_shared_rank(&sh->pub_keep, r);
+    if (r < rank) before += v;
+    all += v;
+  }
+  *my_base = before;
+  base += before;
+  for (int i = lo; i < hi; ++i)
+    if (keep[i]) survivors[base++] = begin + i;
+  __syncthreads();
+  return all;
+}
+
+// Single-CTA pick used for the small top-A choice over the confidence map: marks the A largest of cnt keys
+// in keep[], ties to the lower index.
+__device__ inline void block_top_mark(const uint32_t* keys, uint8_t* keep, int cnt, int A, SelectShared* sh) {
+  const int tid = threadIdx.x, nthr = blockDim.x;
+  const bool keep_all = cnt <= A;
+  uint32_t T = 0;
+  int need_eq = 0;
+  if (!keep_all && A > 0) {
+    uint32_t prefix = 0, mask = 0;
+    int krem = A;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int b = tid; b < 256; b += nthr) sh->tot[b] = 0;
+      __syncthreads();
+      digit_histogram(keys, cnt, mask, prefix, shift, sh->tot);
+      __syncthreads();
+      find_digit(sh->tot, krem, sh);
       __syncthreads();
       prefix |= (uint32_t)sh->digit << shift;
       mask |= 255u << shift;
@@ -84,68 +192,53 @@ __device__ inline int select_core(const uint32_t* keys, uint8_t* flags, uint8_t*
     T = prefix;
     need_eq = krem;
   }
-  // Mark keepers: thread t owns the contiguous positions [t*chunk, (t+1)*chunk).
-  const int chunk = (N + nthr - 1) / nthr;
-  const int lo = min(N, tid * chunk), hi = min(N, lo + chunk);
+  const int chunk = (cnt + nthr - 1) / nthr;
+  const int lo = min(cnt, tid * chunk), hi = min(cnt, lo + chunk);
   int cnt_eq = 0;
-  if (!keep_all && k > 0)
-    for (int i = lo; i < hi; ++i) cnt_eq += ((fl[i] & 3) == 0 && keys[i] == T);
+  if (!keep_all && A > 0)
+    for (int i = lo; i < hi; ++i) cnt_eq += keys[i] == T;
   int tot;
   int eq_rank = block_excl_scan_int(cnt_eq, sh->scan, &tot);
-  int cnt_keep = 0;
   for (int i = lo; i < hi; ++i) {
-    bool keep;
-    if (keep_all) {
-      keep = true;
-    } else if ((fl[i] & 3) != 0) {
-      keep = true;
-    } else if (k <= 0) {
-      keep = false;
-    } else {
-      const uint32_t key = keys[i];
-      keep = key > T || (key == T && eq_rank++ < need_eq);
-    }
-    fl[i] = (uint8_t)((fl[i] & 3) | (keep ? kKeepBit : 0));
-    cnt_keep += keep;
+    bool k = keep_all;
+    if (!keep_all && A > 0) k = keys[i] > T || (keys[i] == T && eq_rank++ < need_eq);
+    keep[i] = k ? 1 : 0;
   }
-  int n_keep;
-  int base = block_excl_scan_int(cnt_keep, sh->scan, &n_keep);
-  for (int i = lo; i < hi; ++i)
-    if (fl[i] & kKeepBit) {
-      if (base < B || keep_all) survivors[base] = i;
-      ++base;
-    }
   __syncthreads();
-  if (!keep_all && n_keep > B) {   // only when |P| > B: keep the first B marked rows
-    if (tid == 0) *bad = 1;
-    n_keep = B;
-  }
-  return n_keep;
 }
 
-// ---- standalone selection over given priorities (one CTA per independent problem)
+// Shared memory a CTA of the selection kernels needs for `span` owned positions (+ np confidence entries).
+__host__ __device__ inline size_t select_smem_bytes(int span, int np) {
+  return ((sizeof(SelectShared) + 15) & ~(size_t)15) + (size_t)span * 4 + 2 * (((size_t)span + 15) & ~(size_t)15) +
+         (size_t)np * 4 + (((size_t)np + 15) & ~(size_t)15) + 16;
+}
+
+// ---- standalone selection over given priorities: one cluster per independent problem (blockIdx.y)
 
 __global__ void __launch_bounds__(kSelectThreads) k_select(const float* __restrict__ r,
                                                            const uint8_t* __restrict__ flags_in, int N, int B,
-                                                           int* __restrict__ survivors, uint32_t* gkeys,
-                                                           int keys_in_smem, int* status) {
+                                                           int* __restrict__ survivors, int* status) {
   extern __shared__ __align__(16) unsigned char smem[];
+  cg::cluster_group cluster = cg::this_cluster();
   SelectShared* sh = reinterpret_cast<SelectShared*>(smem);
   unsigned char* p = smem + ((sizeof(SelectShared) + 15) & ~15);
-  const size_t prob = blockIdx.x;
-  uint32_t* keys = keys_in_smem ? reinterpret_cast<uint32_t*>(p) : gkeys + prob * (size_t)N;
-  if (keys_in_smem) p += (size_t)N * 4;
-  uint8_t* fl = p;
+  const int ncta = (int)cluster.num_blocks();
+  int begin, end;
+  cta_range(N, ncta, (int)cluster.block_rank(), &begin, &end);
+  const int cnt = end - begin, span = (N + ncta - 1) / ncta;
+  uint32_t* keys = reinterpret_cast<uint32_t*>(p);
+  uint8_t* keep = p + (size_t)span * 4;
+  const size_t prob = blockIdx.y;
   const float* rr = r + prob * (size_t)N;
   const uint8_t* ff = flags_in + prob * (size_t)N;
-  for (int i = threadIdx.x; i < N; i += blockDim.x) {
-    keys[i] = rank_key(rr[i]);
-    fl[i] = ff[i] ? 1 : 0;
-  }
+  for (int i = threadIdx.x; i < cnt; i += blockDim.x)
+    keys[i] = ff[begin + i] != 0 ? kKeyProtected : rank_key(rr[begin + i]);
   __syncthreads();
-  int bad = 0;
-  select_core(keys, fl, nullptr, N, B, survivors + prob * (size_t)min(N, B), sh, &bad);
-  if (bad && threadIdx.x == 0 && status) atomicCAS(status, 0, OVGGT_ERR_DEVICE_STATUS);
+  int my_base, bad;
+  const int n_keep = cluster_select(cluster, keys, keep, begin, cnt, N, B, survivors + prob * (size_t)min(N, B), sh,
+                                    &my_base, &bad);
+  if ((bad || n_keep != min(N, B)) && threadIdx.x == 0 && status) atomicCAS(status, 0, OVGGT_ERR_DEVICE_STATUS);
+  cluster.sync();   // no CTA may exit while others still read its shared memory
 }
 
 // ---- the fused per-step kernel
@@ -165,115 +258,149 @@ struct CompressParams {
   const float* override_r;          // [N] or nullptr
   const long long* ids_src; const uint8_t* flags_src; const float* stored_src;   // [N] pre-compaction meta
   long long* ids_dst; uint8_t* flags_dst; float* stored_dst;                     // [<=B] compacted meta
-  float* r_out;                     // [N] priorities as ranked
+  float* r_out;                     // [N] priorities as computed here
   int* survivors;                   // [min(N, B)]
-  uint32_t* gkeys;                  // [N] key scratch when shared memory is too small
-  int keys_in_smem;
   int* status;
   int* n_keep_out;
 };
 
+// Eq. 6 for new-frame token j (aux tokens keep their raw score).
+__device__ __forceinline__ float smoothed_score(const CompressParams& P, int j) {
+  float v = P.s_raw[j];
+  if (j >= P.n_special) {
+    const int q = j - P.n_special, y = q / P.grid_w, x = q - y * P.grid_w;
+    const float* S = P.s_raw + P.n_special;
+    float conv = 0.0f;
+#pragma unroll
+    for (int dy = -1; dy <= 1; ++dy)
+#pragma unroll
+      for (int dx = -1; dx <= 1; ++dx) {
+        const int yy = min(max(y + dy, 0), P.grid_h - 1), xx = min(max(x + dx, 0), P.grid_w - 1);
+        const float w = (dx == 0 && dy == 0) ? P.w_center : ((dx == 0 || dy == 0) ? P.w_edge : P.w_corner);
+        conv = __fmaf_rn(w, S[yy * P.grid_w + xx], conv);
+      }
+    v = __fmaf_rn(P.alpha, conv, __fmul_rn(1.0f - P.alpha, v));
+  }
+  return v;
+}
+
 __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const CompressParams P) {
   extern __shared__ __align__(16) unsigned char smem[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int ncta = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   SelectShared* sh = reinterpret_cast<SelectShared*>(smem);
   unsigned char* p = smem + ((sizeof(SelectShared) + 15) & ~15);
   const int tid = threadIdx.x, nthr = blockDim.x;
   const int n = P.n, M = P.M, N = n + M, Np = P.grid_h * P.grid_w;
-  float* s_new = reinterpret_cast<float*>(p);            // [M] smoothed activation scores
-  p += ((size_t)M * 4 + 15) & ~(size_t)15;
-  uint32_t* keys = P.keys_in_smem ? reinterpret_cast<uint32_t*>(p) : P.gkeys;
-  if (P.keys_in_smem) p += (size_t)N * 4;
-  uint8_t* fl = p;                                       // [N]
-  float* val = reinterpret_cast<float*>(keys);           // values, then priorities, then keys, in place
-  int bad = 0;
+  int begin, end;
+  cta_range(N, ncta, rank, &begin, &end);
+  const int cnt = end - begin, span = (N + ncta - 1) / ncta, span16 = (span + 15) & ~15;
+  uint32_t* keys = reinterpret_cast<uint32_t*>(p);        // [span] values, then the priorities' keys, in place
+  float* val = reinterpret_cast<float*>(keys);
+  uint8_t* fl = p + (size_t)span * 4;                      // [span] protection flags of the owned positions
+  uint8_t* keep = fl + span16;                             // [span]
+  uint32_t* ckeys = reinterpret_cast<uint32_t*>(keep + span16);   // [Np] confidence keys
+  uint8_t* cmark = reinterpret_cast<uint8_t*>(ckeys + Np);        // [Np]
 
-  // -- protection flags (Sec. 3.3)
-  for (int i = tid; i < N; i += nthr) {
-    uint8_t f = P.flags_src[i] & 3;
-    if (i >= n && P.protect_new) f = OVGGT_FLAG_INIT;
-    if (i < n && P.demote_frame >= 0 && f == OVGGT_FLAG_HIST && P.ids_src[i] / M == P.demote_frame)
-      f = OVGGT_FLAG_EVICTABLE;
-    fl[i] = f;
-  }
-  __syncthreads();
-  if (P.register_anchor && P.A > 0) {
-    // the A most confident patch tokens of the new frame, ties to the lower index
-    uint8_t* mark = reinterpret_cast<uint8_t*>(s_new);   // Np <= 4*M bytes, free until smoothing
-    for (int i = tid; i < Np; i += nthr) keys[i] = rank_key(P.conf[i]);
+  // -- anchor registration (Sec. 3.3): the A most confident patch tokens of the new frame, ties to the lower
+  //    index.  Every CTA computes the same marks and uses those of the positions it owns.
+  const bool reg = P.register_anchor && P.A > 0;
+  if (reg) {
+    for (int i = tid; i < Np; i += nthr) ckeys[i] = rank_key(P.conf[i]);
     __syncthreads();
-    const int na = select_core(keys, nullptr, mark, Np, P.A, P.survivors, sh, &bad);
-    __syncthreads();
-    for (int j = tid; j < na; j += nthr) fl[n + P.n_special + P.survivors[j]] = OVGGT_FLAG_HIST;
-    __syncthreads();
+    block_top_mark(ckeys, cmark, Np, P.A, sh);
   }
 
-  // -- Eq. 6 on the patch grid; aux tokens keep their raw score
-  for (int j = tid; j < M; j += nthr) {
-    float v = P.s_raw[j];
-    if (j >= P.n_special) {
-      const int q = j - P.n_special, y = q / P.grid_w, x = q - y * P.grid_w;
-      const float* S = P.s_raw + P.n_special;
-      float conv = 0.0f;
-#pragma unroll
-      for (int dy = -1; dy <= 1; ++dy)
-#pragma unroll
-        for (int dx = -1; dx <= 1; ++dx) {
-          const int yy = min(max(y + dy, 0), P.grid_h - 1), xx = min(max(x + dx, 0), P.grid_w - 1);
-          const float w = (dx == 0 && dy == 0) ? P.w_center : ((dx == 0 || dy == 0) ? P.w_edge : P.w_corner);
-          conv = __fmaf_rn(w, S[yy * P.grid_w + xx], conv);
-        }
-      v = __fmaf_rn(P.alpha, conv, __fmul_rn(1.0f - P.alpha, v));
+  // -- protection flags and values of the owned positions
+  for (int i = tid; i < cnt; i += nthr) {
+    const int g = begin + i;
+    uint8_t f = P.flags_src[g] & 3;
+    float x;
+    if (g >= n) {
+      const int j = g - n;
+      if (P.protect_new) f = OVGGT_FLAG_INIT;
+      if (reg && j >= P.n_special && cmark[j - P.n_special]) f = OVGGT_FLAG_HIST;
+      x = smoothed_score(P, j);
+    } else {
+      if (P.demote_frame >= 0 && f == OVGGT_FLAG_HIST && P.ids_src[g] / M == P.demote_frame) f = OVGGT_FLAG_EVICTABLE;
+      x = (P.mode == OVGGT_SCORE_HYBRID) ? P.d[g] : P.stored_src[g];
     }
-    s_new[j] = v;
+    fl[i] = f;
+    val[i] = x;
   }
   __syncthreads();
 
-  // -- values, then priorities (Eq. 7 or the stored-residual reading)
-  for (int i = tid; i < N; i += nthr)
-    val[i] = i >= n ? s_new[i - n] : (P.mode == OVGGT_SCORE_HYBRID ? P.d[i] : P.stored_src[i]);
-  __syncthreads();
+  // -- Eq. 7: min-max of each group over the whole cluster
   float lo_h = INFINITY, hi_h = -INFINITY, lo_n = INFINITY, hi_n = -INFINITY;
   if (P.mode == OVGGT_SCORE_HYBRID) {
-    for (int i = tid; i < N; i += nthr)
+    for (int i = tid; i < cnt; i += nthr)
       if (fl[i] == 0) {
         const float x = val[i];
-        if (i < n) { lo_h = fminf(lo_h, x); hi_h = fmaxf(hi_h, x); }
-        else       { lo_n = fminf(lo_n, x); hi_n = fmaxf(hi_n, x); }
+        if (begin + i < n) { lo_h = fminf(lo_h, x); hi_h = fmaxf(hi_h, x); }
+        else               { lo_n = fminf(lo_n, x); hi_n = fmaxf(hi_n, x); }
       }
     block_minmax(lo_h, hi_h, sh->fscan, &lo_h, &hi_h);
     block_minmax(lo_n, hi_n, sh->fscan, &lo_n, &hi_n);
+    if (tid == 0) {
+      sh->pub_lo_h = lo_h; sh->pub_hi_h = hi_h; sh->pub_lo_n = lo_n; sh->pub_hi_n = hi_n;
+    }
+    cluster.sync();
+    for (int r = 0; r < ncta; ++r) {
+      const SelectShared* o = cluster.map_shared_rank(sh, r);
+      lo_h = fminf(lo_h, o->pub_lo_h); hi_h = fmaxf(hi_h, o->pub_hi_h);
+      lo_n = fminf(lo_n, o->pub_lo_n); hi_n = fmaxf(hi_n, o->pub_hi_n);
+    }
   }
-  __syncthreads();
-  for (int i = tid; i < N; i += nthr) {
+  for (int i = tid; i < cnt; i += nthr) {
+    const int g = begin + i;
     float r;
+    uint32_t key;
     if (fl[i] != 0) {
       r = INFINITY;
-    } else if (P.mode == OVGGT_SCORE_HYBRID) {
-      const float lo = i < n ? lo_h : lo_n, hi = i < n ? hi_h : hi_n;
-      const float w = i < n ? 1.0f - P.beta : P.beta;
-      r = hi > lo ? __fmul_rn(w, __fdiv_rn(val[i] - lo, hi - lo)) : 0.0f;
+      key = kKeyProtected;
     } else {
-      r = val[i];
+      if (P.mode == OVGGT_SCORE_HYBRID) {
+        const float lo = g < n ? lo_h : lo_n, hi = g < n ? hi_h : hi_n;
+        const float w = g < n ? 1.0f - P.beta : P.beta;
+        r = hi > lo ? __fmul_rn(w, __fdiv_rn(val[i] - lo, hi - lo)) : 0.0f;
+      } else {
+        r = val[i];
+      }
+      key = rank_key(P.override_r ? P.override_r[g] : r);
     }
-    P.r_out[i] = r;                                      // the kernel's own priority, also under teacher forcing
-    if (fl[i] == 0 && P.override_r) r = P.override_r[i];
-    keys[i] = rank_key(r);
+    P.r_out[g] = r;          // the kernel's own priority, also when an override is ranked instead
+    keys[i] = key;
   }
   __syncthreads();
 
   // -- Eq. 8
-  const int n_keep = select_core(keys, fl, nullptr, N, P.B, P.survivors, sh, &bad);
-  __syncthreads();
-  for (int j = tid; j < n_keep; j += nthr) {
-    const int src = P.survivors[j];
-    P.ids_dst[j] = P.ids_src[src];
-    P.flags_dst[j] = fl[src] & 3;
-    P.stored_dst[j] = src >= n ? s_new[src - n] : P.stored_src[src];
+  int my_base, bad;
+  const int n_keep = cluster_select(cluster, keys, keep, begin, cnt, N, P.B, P.survivors, sh, &my_base, &bad);
+
+  // -- compacted meta of this CTA's survivors (order preserved)
+  {
+    const int chunk = (cnt + nthr - 1) / nthr;
+    const int lo = min(cnt, tid * chunk), hi = min(cnt, lo + chunk);
+    int c = 0;
+    for (int i = lo; i < hi; ++i) c += keep[i];
+    int tot;
+    int j = my_base + block_excl_scan_int(c, sh->scan, &tot);
+    for (int i = lo; i < hi; ++i)
+      if (keep[i]) {
+        const int g = begin + i;
+        if (j < P.B) {
+          P.ids_dst[j] = P.ids_src[g];
+          P.flags_dst[j] = fl[i];
+          P.stored_dst[j] = g >= n ? smoothed_score(P, g - n) : P.stored_src[g];
+        }
+        ++j;
+      }
   }
-  if (tid == 0) {
+  if (rank == 0 && tid == 0) {
     *P.n_keep_out = n_keep;
     if (bad || n_keep != min(N, P.B)) atomicCAS(P.status, 0, OVGGT_ERR_DEVICE_STATUS);
   }
+  cluster.sync();   // no CTA may exit while others still read its shared memory
 }
 
 }  // namespace ovggt
