@@ -1,17 +1,20 @@
 // bf16 flash attention for sm_100a: out = softmax(Q K^T / sqrt(64)) V per head, head_dim 64, no mask.
 //
-// One CTA owns one 128-row query tile of one head and a contiguous range of 128-row KV tiles.
-//   warps 0-3   softmax: one thread per query row reads its S row with tcgen05.ld, keeps a running
-//               reference maximum (rescaling O only when the maximum grows by more than 2^8), writes
-//               P as bf16 over the S columns, and at the end normalises and stores O
+// One CTA owns one 128-row query tile of one head and a contiguous range of 128-row KV tiles.  Each KV
+// tile is processed as two 64-row halves with their own S buffer in tensor memory, so the MMAs of one half
+// run while the softmax warps work on the other and the softmax never waits for a whole QK^T -> PV chain.
+//   warps 0-3   softmax: one thread per query row reads its 64 S values of a half with tcgen05.ld, keeps a
+//               running reference maximum (rescaling O only when the maximum grows by more than 2^8),
+//               writes P as bf16 over the first 32 columns of that half, and at the end normalises and stores O
 //   warp 4      TMA producer: Q once, then K and V tiles into 128-byte-swizzled shared-memory stages
-//   warp 5      allocates tensor memory and issues tcgen05.mma:  S = Q K^T  (SS, fp32 in TMEM),
-//               O += P V (P read from TMEM as the A operand, V MN-major from shared memory)
+//   warp 5      allocates tensor memory and issues tcgen05.mma:  S_h = Q K_h^T  (SS, fp32 in TMEM),
+//               O += P_h V_h (P read from TMEM as the A operand, V MN-major from shared memory)
 //   warps 6-7   only complete the second warpgroup, which hands its registers to the softmax warpgroup
-// Two CTAs are resident per SM (256 TMEM columns and ~82 KB shared memory each), so one CTA's MMAs
-// overlap the other's exponentials.  The KV range may be split across CTAs; partial (O, max, sum)
-// triples are merged by a second kernel.  Every mbarrier wait is bounded: on expiry the CTA records
-// OVGGT_ERR_TIMEOUT in the status word and leaves through the common teardown.
+// With head_dim 64 a 128 x 128 tile needs 512 tensor-pipe cycles but 1024 cycles of the 16-per-clock
+// exponential unit, so the exponentials bound the kernel; two CTAs are resident per SM (256 TMEM columns and
+// ~82 KB shared memory each) to keep that unit fed from two independent query tiles.  The KV range may be split
+// across CTAs; partial (O, max, sum) triples are merged by a second kernel.  Every mbarrier wait is bounded: on
+// expiry the CTA records OVGGT_ERR_TIMEOUT in the status word and leaves through the common teardown.
 #pragma once
 
 #include <cuda.h>
@@ -27,13 +30,14 @@ constexpr int kKVStages = 2;
 constexpr int kAttnThreads = 256;
 constexpr int kRegsSoftmax = 216, kRegsOther = 40;   // 2 CTAs x (128 x 216 + 128 x 40) = 64K registers
 constexpr int kTileBytes = kBN * kHD * 2;          // 16 KB
+constexpr int kHalf = kBN / 2;      // KV rows per S buffer
 constexpr int kTmemCols = 256;
-constexpr int kColS = 0, kColO = 128;
+constexpr int kColS = 0, kColO = 128;   // S_0 at columns [0, 64), S_1 at [64, 128), O at [128, 192)
 constexpr float kRescaleThreshold = 8.0f;          // log2 units
 constexpr int kMaxSplits = 16;
 
 struct AttnBarriers {
-  unsigned long long q_full, s_full, p_full, o_full, drain;
+  unsigned long long q_full, s_full[2], p_full[2], pv_done, o_full, drain;
   unsigned long long k_full[kKVStages], k_empty[kKVStages], v_full[kKVStages], v_empty[kKVStages];
   uint32_t tmem_base;
   int abort_flag;
@@ -221,8 +225,11 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
   if (threadIdx.x == 0) {
     mbar_init(&B->q_full, 1);
-    mbar_init(&B->s_full, 1);
-    mbar_init(&B->p_full, 128);
+    for (int hf = 0; hf < 2; ++hf) {
+      mbar_init(&B->s_full[hf], 1);
+      mbar_init(&B->p_full[hf], 128);
+    }
+    mbar_init(&B->pv_done, 1);
     mbar_init(&B->o_full, 1);
     mbar_init(&B->drain, 1);
     for (int s = 0; s < kKVStages; ++s) {
@@ -282,33 +289,59 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     __syncwarp();
   } else if (warp == 5) {
     // ------------------------------------------------ MMA issuer
+    // Issue order (the tensor pipe executes one thread's MMAs in order):
+    //   QK(0,0) QK(0,1) | PV(0,0) QK(1,0) PV(0,1) QK(1,1) | PV(1,0) QK(2,0) PV(1,1) QK(2,1) | ...
+    // QK(t+1,h) overwrites S_h only after PV(t,h) has read P_h from it.
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = idesc_bf16(kBN, false);
+      constexpr uint32_t idesc_qk = idesc_bf16(kHalf, false);
       constexpr uint32_t idesc_pv = idesc_bf16(kHD, true);
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ));
-      bool ok = mbar_wait(&B->q_full, 0, B, P.status);
-      for (int it = 0; it < n_tiles && ok; ++it) {
-        const int s = it % kKVStages;
-        const uint32_t ph = (uint32_t)(it / kKVStages) & 1u;
-        ok = mbar_wait(&B->k_full[s], ph, B, P.status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint64_t dk = smem_desc_sw128(smem_u32(sK + s * kTileBytes));
+      // S_hf = Q K_hf^T for the KV tile held in stage `st` (64 rows = 8 swizzle groups = 8192 bytes per half)
+      auto issue_qk = [&](int st, int hf) {
+        const uint64_t dk = smem_desc_sw128(smem_u32(sK + st * kTileBytes + hf * (kTileBytes / 2)));
 #pragma unroll
         for (int kk = 0; kk < kHD / 16; ++kk)     // 16 elements of head dim = 32 bytes inside the swizzled row
-          mma_ss(tmem + kColS, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_qk, kk > 0);
-        tc_commit(&B->k_empty[s]);
-        tc_commit(&B->s_full);
-        ok = mbar_wait(&B->p_full, (uint32_t)it & 1u, B, P.status);
-        if (!ok) break;
+          mma_ss(tmem + kColS + hf * kHalf, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_qk, kk > 0);
+      };
+      bool ok = mbar_wait(&B->q_full, 0, B, P.status);
+      if (ok) ok = mbar_wait(&B->k_full[0], 0, B, P.status);
+      if (ok) {
+        tc_fence_after();
+        issue_qk(0, 0);
+        tc_commit(&B->s_full[0]);
+        issue_qk(0, 1);
+        tc_commit(&B->s_full[1]);
+        tc_commit(&B->k_empty[0]);
+      }
+      for (int it = 0; it < n_tiles && ok; ++it) {
+        const int s = it % kKVStages, s1 = (it + 1) % kKVStages;
+        const uint32_t ph = (uint32_t)(it / kKVStages) & 1u, ph1 = (uint32_t)((it + 1) / kKVStages) & 1u;
+        const bool more = it + 1 < n_tiles;
         ok = mbar_wait(&B->v_full[s], ph, B, P.status);
         if (!ok) break;
-        tc_fence_after();
         const uint64_t dv = smem_desc_sw128(smem_u32(sV + s * kTileBytes));
 #pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk)     // 16 KV rows = 2048 bytes; P: 8 TMEM columns per 16 bf16
-          mma_ts(tmem + kColO, tmem + kColS + kk * 8, dv + (uint64_t)(kk * 128), idesc_pv, (it > 0 || kk > 0));
-        tc_commit(&B->v_empty[s]);
+        for (int hf = 0; hf < 2; ++hf) {
+          ok = mbar_wait(&B->p_full[hf], (uint32_t)it & 1u, B, P.status);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < kHalf / 16; ++kk)   // 16 KV rows = 2048 bytes; P: 8 TMEM columns per 16 bf16
+            mma_ts(tmem + kColO, tmem + kColS + hf * kHalf + kk * 8, dv + (uint64_t)((hf * (kHalf / 16) + kk) * 128),
+                   idesc_pv, (it > 0 || hf > 0 || kk > 0));
+          if (hf == 1) tc_commit(&B->v_empty[s]);
+          tc_commit(&B->pv_done);
+          if (more) {
+            if (hf == 0) {
+              ok = mbar_wait(&B->k_full[s1], ph1, B, P.status);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            issue_qk(s1, hf);
+            tc_commit(&B->s_full[hf]);
+            if (hf == 1) tc_commit(&B->k_empty[s1]);
+          }
+        }
       }
       if (ok) {
         tc_commit(&B->o_full);
@@ -329,35 +362,40 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const float c = 1.4426950408889634f * 0.125f;     // log2(e) / sqrt(64)
     float mref = 0.0f, l = 0.0f;
     bool ok = true;
-    for (int it = 0; it < n_tiles; ++it) {
-      ok = mbar_wait(&B->s_full, (uint32_t)it & 1u, B, P.status);
+    for (int idx = 0; idx < 2 * n_tiles; ++idx) {       // idx = 2 * tile + half
+      const int it = idx >> 1, hf = idx & 1;
+      ok = mbar_wait(&B->s_full[hf], (uint32_t)it & 1u, B, P.status);
       if (!ok) break;
       tc_fence_after();
-      uint32_t s[128];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) tmem_ld32(t_row + kColS + j * 32, s + j * 32);
+      uint32_t s[kHalf];
+      tmem_ld32(t_row + kColS + hf * kHalf, s);
+      tmem_ld32(t_row + kColS + hf * kHalf + 32, s + 32);
       tmem_wait_ld();
-      const int col0 = (t_begin + it) * kBN;
-      if (col0 + kBN > P.N) {
+      const int col0 = (t_begin + it) * kBN + hf * kHalf;
+      if (col0 + kHalf > P.N) {
 #pragma unroll
-        for (int j = 0; j < 128; ++j)
+        for (int j = 0; j < kHalf; ++j)
           if (col0 + j >= P.N) s[j] = 0xFF800000u;     // -inf on columns past the last row
       }
       // row maximum: four independent chains of 3-input maxima
       float m4[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        m4[q] = fmaxf(__uint_as_float(s[32 * q]), __uint_as_float(s[32 * q + 1]));
+        m4[q] = fmaxf(__uint_as_float(s[16 * q]), __uint_as_float(s[16 * q + 1]));
 #pragma unroll
-        for (int j = 2; j < 32; j += 2)
-          m4[q] = max3(m4[q], __uint_as_float(s[32 * q + j]), __uint_as_float(s[32 * q + j + 1]));
+        for (int j = 2; j < 16; j += 2)
+          m4[q] = max3(m4[q], __uint_as_float(s[16 * q + j]), __uint_as_float(s[16 * q + j + 1]));
       }
       float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * c;
-      if (it == 0) {
+      if (idx == 0) {
         mref = mx;
       } else {
         const bool grow = mx - mref > kRescaleThreshold;
         if (__any_sync(0xFFFFFFFFu, grow)) {
+          // O may still be accumulating the previous half: PV(idx - 1) is the (idx - 1)-th phase of pv_done
+          ok = mbar_wait(&B->pv_done, (uint32_t)(idx - 1) & 1u, B, P.status);
+          if (!ok) break;
+          tc_fence_after();
           const float a = grow ? ex2(mref - mx) : 1.0f;
           if (grow) {
             mref = mx;
@@ -380,7 +418,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
       for (int q = 0; q < 4; ++q) acc[q] = make_float2(0.0f, 0.0f);
 #pragma unroll
-      for (int j = 0; j < 128; j += 2) {
+      for (int j = 0; j < kHalf; j += 2) {
         const float2 x = fma2(make_float2(__uint_as_float(s[j]), __uint_as_float(s[j + 1])), c2, nm2);
         const float2 p = make_float2(ex2(x.x), ex2(x.y));
         acc[(j >> 1) & 3] = add2(acc[(j >> 1) & 3], p);
@@ -388,11 +426,10 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       const float2 t = add2(add2(acc[0], acc[1]), add2(acc[2], acc[3]));
       l += t.x + t.y;
-      tmem_st32(t_row + kColS, s);
-      tmem_st32(t_row + kColS + 32, s + 32);
+      tmem_st32(t_row + kColS + hf * kHalf, s);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&B->p_full);
+      mbar_arrive(&B->p_full[hf]);
     }
     if (ok) ok = mbar_wait(&B->o_full, 0, B, P.status);
     if (ok) {
