@@ -27,8 +27,10 @@ struct SelectShared {
   int scan[64];
   float fscan[64];
   int digit, krem;
-  int pub_eq, pub_keep;      // this CTA's totals, read by the other CTAs of the cluster
+  int pub_gt, pub_eq;        // this CTA's counts of keys above / equal to the threshold, read by the cluster
   float pub_lo_h, pub_hi_h, pub_lo_n, pub_hi_n;
+  int all_gt[kSelectMaxCtas], all_eq[kSelectMaxCtas];   // the whole cluster's counts, gathered by one warp
+  float mm[4];               // cluster-wide lo_h, hi_h, lo_n, hi_n
 };
 
 // Range of positions owned by CTA `rank` when N positions are split over `ncta` CTAs.
@@ -124,19 +126,44 @@ __device__ inline int cluster_select(cg::cluster_group& cluster, const uint32_t*
   // Thread t owns the contiguous local positions [t*chunk, (t+1)*chunk).
   const int chunk = (cnt + nthr - 1) / nthr;
   const int lo = min(cnt, tid * chunk), hi = min(cnt, lo + chunk);
-  int cnt_eq = 0;
-  if (!keep_all)
-    for (int i = lo; i < hi; ++i) cnt_eq += keys[i] == T;
-  int eq_total;
-  int eq_rank = block_excl_scan_int(cnt_eq, sh->scan, &eq_total);
-  if (tid == 0) sh->pub_eq = eq_total;
-  cluster.sync();
-  int eq_all = 0;
-  for (int r = 0; r < ncta; ++r) {
-    const int v = *cluster.map_shared_rank(&sh->pub_eq, r);
-    if (r < rank) eq_rank += v;
-    eq_all += v;
+  // One exchange settles everything: with (keys above T, keys equal to T) of every CTA, each CTA knows how
+  // many of its ties are admitted (ties go to the lower position, i.e. to the lower rank first) and where its
+  // survivors start in the output.
+  int cnt_gt = 0, cnt_eq = 0;
+  if (keep_all) {
+    cnt_gt = hi - lo;
+  } else {
+    for (int i = lo; i < hi; ++i) {
+      const uint32_t key = keys[i];
+      cnt_gt += key > T;
+      cnt_eq += key == T;
+    }
   }
+  int gt_total, eq_total;
+  block_excl_scan_int(cnt_gt, sh->scan, &gt_total);
+  int eq_rank = block_excl_scan_int(cnt_eq, sh->scan, &eq_total);   // ties before this thread's, within the CTA
+  if (tid == 0) {
+    sh->pub_gt = gt_total;
+    sh->pub_eq = eq_total;
+  }
+  cluster.sync();
+  if (tid < ncta) {                                   // one remote read per lane instead of ncta per thread
+    sh->all_gt[tid] = *cluster.map_shared_rank(&sh->pub_gt, tid);
+    sh->all_eq[tid] = *cluster.map_shared_rank(&sh->pub_eq, tid);
+  }
+  __syncthreads();
+  int before = 0, all = 0, eq_before = 0, eq_all = 0;
+  for (int r = 0; r < ncta; ++r) {
+    const int e = sh->all_eq[r], gcount = sh->all_gt[r];
+    const int adm = keep_all ? 0 : max(0, min(e, need_eq - eq_all));   // ties of rank r that are admitted
+    if (r < rank) {
+      before += gcount + adm;
+      eq_before += e;
+    }
+    all += gcount + adm;
+    eq_all += e;
+  }
+  eq_rank += eq_before;
   // more protected rows than the budget holds: only the first B of them can stay
   *bad = (!keep_all && T == kKeyProtected && eq_all > need_eq) ? 1 : 0;
   int cnt_keep = 0;
@@ -151,14 +178,6 @@ __device__ inline int cluster_select(cg::cluster_group& cluster, const uint32_t*
   }
   int keep_total;
   int base = block_excl_scan_int(cnt_keep, sh->scan, &keep_total);
-  if (tid == 0) sh->pub_keep = keep_total;
-  cluster.sync();
-  int before = 0, all = 0;
-  for (int r = 0; r < ncta; ++r) {
-    const int v = *cluster.map_shared_rank(&sh->pub_keep, r);
-    if (r < rank) before += v;
-    all += v;
-  }
   *my_base = before;
   base += before;
   for (int i = lo; i < hi; ++i)
@@ -256,7 +275,7 @@ struct CompressParams {
   const float* d;                   // [n] key diversity (hybrid mode)
   const float* conf;                // [grid_h*grid_w]
   const float* override_r;          // [N] or nullptr
-  const long long* ids_src; const uint8_t* flags_src; const float* stored_src;   // [N] pre-compaction meta
+  const long long* ids_src; const uint8_t* flags_src; float* stored_src;         // [N] pre-compaction meta (stored: new rows filled here)
   long long* ids_dst; uint8_t* flags_dst; float* stored_dst;                     // [<=B] compacted meta
   float* r_out;                     // [N] priorities as computed here
   int* survivors;                   // [min(N, B)]
@@ -321,6 +340,7 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
       if (P.protect_new) f = OVGGT_FLAG_INIT;
       if (reg && j >= P.n_special && cmark[j - P.n_special]) f = OVGGT_FLAG_HIST;
       x = smoothed_score(P, j);
+      P.stored_src[g] = x;       // the score the row keeps (read back below by the same CTA when the row survives)
     } else {
       if (P.demote_frame >= 0 && f == OVGGT_FLAG_HIST && P.ids_src[g] / M == P.demote_frame) f = OVGGT_FLAG_EVICTABLE;
       x = (P.mode == OVGGT_SCORE_HYBRID) ? P.d[g] : P.stored_src[g];
@@ -345,11 +365,23 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
       sh->pub_lo_h = lo_h; sh->pub_hi_h = hi_h; sh->pub_lo_n = lo_n; sh->pub_hi_n = hi_n;
     }
     cluster.sync();
-    for (int r = 0; r < ncta; ++r) {
-      const SelectShared* o = cluster.map_shared_rank(sh, r);
-      lo_h = fminf(lo_h, o->pub_lo_h); hi_h = fmaxf(hi_h, o->pub_hi_h);
-      lo_n = fminf(lo_n, o->pub_lo_n); hi_n = fmaxf(hi_n, o->pub_hi_n);
+    if (tid < 32) {                                   // one warp gathers: lane r reads CTA r's four values
+      float a = INFINITY, b = -INFINITY, c2 = INFINITY, d2 = -INFINITY;
+      if (tid < ncta) {
+        const SelectShared* o = cluster.map_shared_rank(sh, tid);
+        a = o->pub_lo_h; b = o->pub_hi_h; c2 = o->pub_lo_n; d2 = o->pub_hi_n;
+      }
+#pragma unroll
+      for (int off = 4; off > 0; off >>= 1) {         // kSelectMaxCtas = 8 lanes carry values
+        a = fminf(a, __shfl_xor_sync(0xFFFFFFFFu, a, off));
+        b = fmaxf(b, __shfl_xor_sync(0xFFFFFFFFu, b, off));
+        c2 = fminf(c2, __shfl_xor_sync(0xFFFFFFFFu, c2, off));
+        d2 = fmaxf(d2, __shfl_xor_sync(0xFFFFFFFFu, d2, off));
+      }
+      if (tid == 0) { sh->mm[0] = a; sh->mm[1] = b; sh->mm[2] = c2; sh->mm[3] = d2; }
     }
+    __syncthreads();
+    lo_h = sh->mm[0]; hi_h = sh->mm[1]; lo_n = sh->mm[2]; hi_n = sh->mm[3];
   }
   for (int i = tid; i < cnt; i += nthr) {
     const int g = begin + i;
@@ -391,7 +423,7 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
         if (j < P.B) {
           P.ids_dst[j] = P.ids_src[g];
           P.flags_dst[j] = fl[i];
-          P.stored_dst[j] = g >= n ? smoothed_score(P, g - n) : P.stored_src[g];
+          P.stored_dst[j] = P.stored_src[g];
         }
         ++j;
       }
