@@ -35,6 +35,64 @@ __global__ void __launch_bounds__(256) k_compact(const uint4* __restrict__ k_src
   }
 }
 
+constexpr int kCompactSumMaxVec = 128;   // rows of up to 128 16-byte vectors (C <= 1024 bf16) in the fused variant
+
+// The same gather that also sums, per CTA, the columns of the K rows it writes: part[blockIdx.x, c] = sum of
+// k_dst[j, c] over this CTA's K rows, each warp folding its rows in item order and the CTA folding its four
+// K warps in warp order (the warps of a CTA alternate between K and V items because the total number of warps
+// is even).  The sums over all CTAs are the column sums of the compacted keys: the centroid the next step's
+// diversity score needs, obtained without another pass over K.  Requires nvec <= kCompactSumMaxVec.
+template <int DT>
+__global__ void __launch_bounds__(256) k_compact_colsum(const uint4* __restrict__ k_src, const uint4* __restrict__ v_src,
+                                                        const int* __restrict__ survivors, int n_keep, int nvec,
+                                                        uint4* __restrict__ k_dst, uint4* __restrict__ v_dst,
+                                                        float* __restrict__ part) {
+  constexpr int VEC = VecOf<DT>::n;
+  __shared__ float red[4][kCompactSumMaxVec * VEC];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
+  float acc[4][VEC];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[i][e] = 0.0f;
+  for (int item = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5); item < 2 * n_keep;
+       item += warps_total) {
+    const int j = item >> 1;
+    const int src = survivors[j];
+    if (item & 1) {
+      warp_copy_row(v_src + (size_t)src * nvec, v_dst + (size_t)j * nvec, nvec, lane);
+    } else {
+      const uint4* sp = k_src + (size_t)src * nvec;
+      uint4* dp = k_dst + (size_t)j * nvec;
+      uint4 u[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (lane + 32 * i < nvec) u[i] = ld_nc(sp + lane + 32 * i);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (lane + 32 * i < nvec) {
+          dp[lane + 32 * i] = u[i];
+          float f[VEC];
+          unpack<DT>(u[i], f);
+#pragma unroll
+          for (int e = 0; e < VEC; ++e) acc[i][e] += f[e];
+        }
+    }
+  }
+  if ((warp & 1) == 0) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (lane + 32 * i < nvec)
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) red[warp >> 1][(lane + 32 * i) * VEC + e] = acc[i][e];
+  }
+  __syncthreads();
+  const int C = nvec * VEC;
+  for (int c = threadIdx.x; c < C; c += blockDim.x)
+    part[(size_t)blockIdx.x * C + c] = ((red[0][c] + red[1][c]) + red[2][c]) + red[3][c];
+}
+
 // Rows [n, n+M) of the cache := the frame's K and V; their meta: ids frame*M + j, evictable, score 0.
 __global__ void __launch_bounds__(256) k_append(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
                                                 int M, int nvec, int n, long long frame_id,

@@ -97,9 +97,46 @@ int launch_diversity(const void* K, int rows, int C, int dtype, float* part, flo
   LAUNCHED();
   const int grid = std::min((rows + 7) / 8, 148 * 8);
   const size_t smem = (size_t)C * 4;
-  if (dtype == kBF16) k_diversity<kBF16><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, d);
-  else                k_diversity<kF32><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, d);
+  if (dtype == kBF16) k_diversity<kBF16><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d);
+  else                k_diversity<kF32><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d);
   LAUNCHED();
+  return OVGGT_OK;
+}
+
+constexpr int kColsumSlices = 8;
+
+// Diversity from the per-CTA column sums the last compaction left (nparts rows of part): no pass over K for the sums.
+// slices: [kColsumSlices, C] floats.
+int launch_diversity_from_parts(const void* K, int rows, int C, int dtype, const float* part, int nparts, float* slices,
+                                float* d, cudaStream_t st) {
+  if (rows <= 0) return OVGGT_OK;
+  const int nvec = C * elem_bytes(dtype) / 16;
+  k_colsum_final_sliced<<<dim3((C + 31) / 32, kColsumSlices), 1024, 0, st>>>(part, nparts, C, slices);
+  LAUNCHED();
+  // every CTA first folds the slices (kColsumSlices x C floats): keep that a small share of its work
+  const int grid = std::min((rows + 63) / 64, 148 * 8);
+  const size_t smem = (size_t)C * 4;
+  if (dtype == kBF16) k_diversity<kBF16><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, slices, kColsumSlices, d);
+  else                k_diversity<kF32><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, slices, kColsumSlices, d);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
+// Compaction that also leaves per-CTA column sums of the keys it writes; *nparts = number of partial rows written.
+int launch_compact_colsum(const void* ks, const void* vs, const int* surv, int n_keep, int C, int dtype, void* kd,
+                          void* vd, float* part, int* nparts, cudaStream_t st) {
+  *nparts = 0;
+  if (n_keep <= 0) return OVGGT_OK;
+  const int nvec = C * elem_bytes(dtype) / 16;
+  const int grid = std::min((2 * n_keep + 7) / 8, 148 * 8);
+  if (dtype == kBF16)
+    k_compact_colsum<kBF16><<<grid, 256, 0, st>>>((const uint4*)ks, (const uint4*)vs, surv, n_keep, nvec, (uint4*)kd,
+                                                  (uint4*)vd, part);
+  else
+    k_compact_colsum<kF32><<<grid, 256, 0, st>>>((const uint4*)ks, (const uint4*)vs, surv, n_keep, nvec, (uint4*)kd,
+                                                 (uint4*)vd, part);
+  LAUNCHED();
+  *nparts = grid;
   return OVGGT_OK;
 }
 
@@ -148,6 +185,8 @@ struct LayerState {
   float *s_raw, *d, *r;
   int* surv;
   int* n_keep_dev;
+  float* colsum_part = nullptr;   // [148 * 8, C]: per-CTA column sums of the keys the last compaction wrote
+  int colsum_nparts = 0;          // 0: not available (the next step sums the keys itself)
   size_t kv_bytes = 0;
 };
 
@@ -246,7 +285,7 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
   for (int l = 0; l < c->n_layers; ++l) {
     const size_t R = (size_t)c->budget[l] + M;
     max_rows = std::max(max_rows, (int)R);
-    size_t off[16];
+    size_t off[20];
     int i = 0;
     for (int b = 0; b < 2; ++b) off[i++] = L.take(R * C * eb);
     for (int b = 0; b < 2; ++b) off[i++] = L.take(R * C * eb);
@@ -258,6 +297,7 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
     off[i++] = L.take(R * 4);           // r
     off[i++] = L.take(R * 4);           // survivors
     off[i++] = L.take(64);              // n_keep
+    off[i++] = L.take((size_t)148 * 8 * C * 4);   // column-sum partials of the compaction
     if (h) {
       LayerState& S = h->layers[l];
       i = 0;
@@ -271,12 +311,13 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
       S.r = reinterpret_cast<float*>(base + off[i++]);
       S.surv = reinterpret_cast<int*>(base + off[i++]);
       S.n_keep_dev = reinterpret_cast<int*>(base + off[i++]);
+      S.colsum_part = reinterpret_cast<float*>(base + off[i++]);
       S.budget = c->budget[l];
       S.kv_bytes = 4 * R * C * eb;
     }
   }
   const size_t o_part = L.take((size_t)kMaxColsumParts * C * 4);
-  const size_t o_ksum = L.take((size_t)C * 4);
+  const size_t o_ksum = L.take((size_t)kColsumSlices * C * 4);
   const size_t o_attn = L.take(ovggt_k_attention_scratch_bytes(M, max_rows, c->n_heads));
   const size_t o_status = L.take(64);
   size_t o_stage[5];
@@ -430,7 +471,10 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
   if (rc) return rc;
   if (c.score_mode == OVGGT_SCORE_HYBRID && n > 0) {
     ProfScope ps(h, OVGGT_PROF_DIVERSITY, st);
-    rc = launch_diversity(S.kbuf[b], n, C, c.dtype, h->colsum_part, h->ksum, S.d, st);
+    if (S.colsum_nparts > 0)
+      rc = launch_diversity_from_parts(S.kbuf[b], n, C, c.dtype, S.colsum_part, S.colsum_nparts, h->ksum, S.d, st);
+    else
+      rc = launch_diversity(S.kbuf[b], n, C, c.dtype, h->colsum_part, h->ksum, S.d, st);
     if (rc) return rc;
   }
   CompressParams P;
@@ -460,7 +504,13 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
   const int n_keep = std::min(N, B);
   {
     ProfScope ps(h, OVGGT_PROF_COMPACT, st);
-    rc = launch_compact(S.kbuf[b], S.vbuf[b], S.surv, n_keep, C, c.dtype, S.kbuf[b ^ 1], S.vbuf[b ^ 1], st);
+    const bool fuse = c.score_mode == OVGGT_SCORE_HYBRID && C * h->elem / 16 <= kCompactSumMaxVec;
+    S.colsum_nparts = 0;
+    if (fuse)
+      rc = launch_compact_colsum(S.kbuf[b], S.vbuf[b], S.surv, n_keep, C, c.dtype, S.kbuf[b ^ 1], S.vbuf[b ^ 1],
+                                 S.colsum_part, &S.colsum_nparts, st);
+    else
+      rc = launch_compact(S.kbuf[b], S.vbuf[b], S.surv, n_keep, C, c.dtype, S.kbuf[b ^ 1], S.vbuf[b ^ 1], st);
   }
   if (rc) return rc;
 
@@ -581,6 +631,7 @@ extern "C" int ovggt_cache_import(ovggt_cache* h, int32_t layer, const int64_t* 
     CK(cudaMemcpy(S.vbuf[b], v, (size_t)n * row, cudaMemcpyHostToDevice));
   }
   S.n = n;
+  S.colsum_nparts = 0;          // the imported keys have not been summed
   S.pending = false;
   S.n_prot_init = n_init;
   S.n_prot_hist = n_hist;

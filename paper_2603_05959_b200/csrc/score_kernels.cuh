@@ -93,16 +93,42 @@ __global__ void __launch_bounds__(1024) k_colsum_final(const float* __restrict__
   }
 }
 
+// Stage 2 for many partials (the compaction kernel leaves one per CTA): CTA (x, y) folds the partials
+// p = y, y + gridDim.y, ... of its 32 columns the same way; ksum8[y, c] holds the result and the diversity kernel
+// folds the gridDim.y slices in order when it stages the sums.
+__global__ void __launch_bounds__(1024) k_colsum_final_sliced(const float* __restrict__ part, int nparts, int C,
+                                                              float* __restrict__ ksum_slices) {
+  __shared__ float sh[32][33];
+  const int cx = threadIdx.x & 31, py = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + cx;
+  float acc = 0.0f;
+  if (c < C)
+    for (int p = blockIdx.y + py * gridDim.y; p < nparts; p += 32 * gridDim.y) acc += part[(size_t)p * C + c];
+  sh[py][cx] = acc;
+  __syncthreads();
+  if (py == 0 && c < C) {
+    float t = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) t += sh[i][cx];
+    ksum_slices[(size_t)blockIdx.y * C + c] = t;
+  }
+}
+
 // d[row] = 1 - (k_row . ksum) / (|k_row| |ksum|); the cosine with the centroid equals the cosine
 // with the column sum.  A zero vector has cosine 0.  One warp per row, ksum staged in shared memory;
 // |ksum|^2 is folded by every warp in the same order, so all CTAs agree on it.
 template <int DT>
 __global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, int rows, int nvec,
-                                                   const float* __restrict__ ksum, float* __restrict__ d) {
+                                                   const float* __restrict__ ksum, int n_slices,
+                                                   float* __restrict__ d) {
   constexpr int VEC = VecOf<DT>::n;
   extern __shared__ float sh_ksum[];
   const int C = nvec * VEC;
-  for (int c = threadIdx.x; c < C; c += blockDim.x) sh_ksum[c] = ksum[c];
+  for (int c = threadIdx.x; c < C; c += blockDim.x) {   // ksum: [n_slices, C], folded in slice order
+    float t = ksum[c];
+    for (int sl = 1; sl < n_slices; ++sl) t += ksum[(size_t)sl * C + c];
+    sh_ksum[c] = t;
+  }
   __syncthreads();
   const int lane = threadIdx.x & 31;
   float kn = 0.0f;
