@@ -113,8 +113,7 @@ int launch_diversity_from_parts(const void* K, int rows, int C, int dtype, const
   const int nvec = C * elem_bytes(dtype) / 16;
   k_colsum_final_sliced<<<dim3((C + 31) / 32, kColsumSlices), 1024, 0, st>>>(part, nparts, C, slices);
   LAUNCHED();
-  // every CTA first folds the slices (kColsumSlices x C floats): keep that a small share of its work
-  const int grid = std::min((rows + 63) / 64, 148 * 8);
+  const int grid = std::min((rows + 15) / 16, 148 * 8);
   const size_t smem = (size_t)C * 4;
   if (dtype == kBF16) k_diversity<kBF16><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, slices, kColsumSlices, d);
   else                k_diversity<kF32><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, slices, kColsumSlices, d);

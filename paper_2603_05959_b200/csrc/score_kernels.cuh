@@ -102,8 +102,10 @@ __global__ void __launch_bounds__(1024) k_colsum_final_sliced(const float* __res
   const int cx = threadIdx.x & 31, py = threadIdx.x >> 5;
   const int c = blockIdx.x * 32 + cx;
   float acc = 0.0f;
-  if (c < C)
+  if (c < C) {
+#pragma unroll 8
     for (int p = blockIdx.y + py * gridDim.y; p < nparts; p += 32 * gridDim.y) acc += part[(size_t)p * C + c];
+  }
   sh[py][cx] = acc;
   __syncthreads();
   if (py == 0 && c < C) {
@@ -137,34 +139,44 @@ __global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, 
     for (int e = 0; e < VEC; ++e) kn = __fmaf_rn(sh_ksum[v * VEC + e], sh_ksum[v * VEC + e], kn);
   kn = warp_sum(kn);
   const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
-  for (int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5); row < rows;
-       row += warps_total) {
-    const uint4* p = K + (size_t)row * nvec;
-    float dot = 0.0f, nrm = 0.0f;
+  // two rows per iteration, so that eight 16-byte loads per lane are in flight
+  for (int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5) * 2; row < rows;
+       row += 2 * warps_total) {
+    const bool two = row + 1 < rows;
+    const uint4* p0 = K + (size_t)row * nvec;
+    const uint4* p1 = p0 + (two ? nvec : 0);
+    float dot[2] = {0.0f, 0.0f}, nrm[2] = {0.0f, 0.0f};
     for (int v0 = lane; v0 < nvec; v0 += 128) {
-      uint4 u[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (v0 + 32 * i < nvec) u[i] = ld_nc(p + v0 + 32 * i);
+      uint4 u[2][4];
 #pragma unroll
       for (int i = 0; i < 4; ++i)
         if (v0 + 32 * i < nvec) {
-          float f[VEC];
-          unpack<DT>(u[i], f);
-          const float* ks = sh_ksum + (v0 + 32 * i) * VEC;
-#pragma unroll
-          for (int e = 0; e < VEC; ++e) {
-            dot = __fmaf_rn(f[e], ks[e], dot);
-            nrm = __fmaf_rn(f[e], f[e], nrm);
-          }
+          u[0][i] = ld_nc(p0 + v0 + 32 * i);
+          u[1][i] = ld_nc(p1 + v0 + 32 * i);
         }
+#pragma unroll
+      for (int r = 0; r < 2; ++r)
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (v0 + 32 * i < nvec) {
+            float f[VEC];
+            unpack<DT>(u[r][i], f);
+            const float* ks = sh_ksum + (v0 + 32 * i) * VEC;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+              dot[r] = __fmaf_rn(f[e], ks[e], dot[r]);
+              nrm[r] = __fmaf_rn(f[e], f[e], nrm[r]);
+            }
+          }
     }
-    dot = warp_sum(dot);
-    nrm = warp_sum(nrm);
-    if (lane == 0) {
-      float cosv = 0.0f;
-      if (nrm > 0.0f && kn > 0.0f) cosv = __fdiv_rn(dot, __fmul_rn(__fsqrt_rn(nrm), __fsqrt_rn(kn)));
-      d[row] = 1.0f - cosv;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      const float dt = warp_sum(dot[r]), nr = warp_sum(nrm[r]);
+      if (lane == 0 && (r == 0 || two)) {
+        float cosv = 0.0f;
+        if (nr > 0.0f && kn > 0.0f) cosv = __fdiv_rn(dt, __fmul_rn(__fsqrt_rn(nr), __fsqrt_rn(kn)));
+        d[row + r] = 1.0f - cosv;
+      }
     }
   }
 }
