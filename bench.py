@@ -140,37 +140,49 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------- CPU oracle leg
 
-def oracle_rate(cfg: gen.StreamConfig, frames: int, attn_rows: int, threads: int) -> dict:
-    """Frames/s of the CPU oracle as it stands, at steady state.  The cache is filled with append +
-    compress only (untimed); then `frames` frames are timed: selection path in full, dense attention on
-    `attn_rows` sampled query rows x all heads, scaled to the M rows of a frame."""
-    from oracle import oracle as orc
-    orc.set_threads(threads)
-    layer = orc.OracleLayer.from_stream(cfg)
-    M = cfg.tokens_per_frame
-    t = 0
-    while layer.n_rows < cfg.budget:
-        fi = gen.frame_inputs(cfg, t)
-        layer.attend(t, fi.q, fi.k, fi.v, compute=False)
-        layer.compress(fi.resid, fi.conf, fi.rho)
-        t += 1
-    rows = np.sort(np.random.default_rng(cfg.seed).choice(M, min(attn_rows, M), replace=False)).astype(np.int32)
-    t_attn = t_comp = 0.0
-    for _ in range(frames):
-        fi = gen.frame_inputs(cfg, t)
+class OracleRunner:
+    """The CPU oracle as it stands, at steady state: the cache is filled with append + compress only (untimed);
+    each timed frame runs the selection path in full and dense attention on `attn_rows` sampled query rows x all
+    heads, whose time is scaled to the M rows of a frame."""
+
+    def __init__(self, cfg: gen.StreamConfig, attn_rows: int, threads: int):
+        from oracle import oracle as orc
+        orc.set_threads(threads)
+        self.cfg, self.threads = cfg, threads
+        self.layer = orc.OracleLayer.from_stream(cfg)
+        self.M = cfg.tokens_per_frame
+        self.t = 0
+        while self.layer.n_rows < cfg.budget:
+            fi = gen.frame_inputs(cfg, self.t)
+            self.layer.attend(self.t, fi.q, fi.k, fi.v, compute=False)
+            self.layer.compress(fi.resid, fi.conf, fi.rho)
+            self.t += 1
+        self.rows = np.sort(np.random.default_rng(cfg.seed).choice(self.M, min(attn_rows, self.M),
+                                                                    replace=False)).astype(np.int32)
+        self.measured = 0.0
+
+    def frame(self) -> float:
+        """One frame; returns its extrapolated seconds."""
+        fi = gen.frame_inputs(self.cfg, self.t)
         a = time.perf_counter()
-        layer.attend(t, fi.q, fi.k, fi.v, rows=rows)
+        self.layer.attend(self.t, fi.q, fi.k, fi.v, rows=self.rows)
         b = time.perf_counter()
-        layer.compress(fi.resid, fi.conf, fi.rho)
+        self.layer.compress(fi.resid, fi.conf, fi.rho)
         c = time.perf_counter()
-        t_attn += b - a
-        t_comp += c - b
-        t += 1
-    per_frame = (t_attn * (M / len(rows)) + t_comp) / frames
-    return {"value": 1.0 / per_frame, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": f"{frames} steady-state frames; selection path in full, dense attention on {len(rows)} of {M} "
-                      f"query rows x all heads, attention time scaled by {M}/{len(rows)} (extrapolated)",
-            "measured_seconds": t_attn + t_comp, "ms_per_frame_extrapolated": per_frame * 1e3}
+        self.t += 1
+        self.measured += c - a
+        return (b - a) * (self.M / len(self.rows)) + (c - b)
+
+    def sample(self, frames: int) -> str:
+        return (f"{frames} steady-state frames; selection path in full, dense attention on {len(self.rows)} of "
+                f"{self.M} query rows x all heads, attention time scaled by {self.M}/{len(self.rows)} (extrapolated)")
+
+
+def oracle_rate(cfg: gen.StreamConfig, frames: int, attn_rows: int, threads: int) -> dict:
+    run = OracleRunner(cfg, attn_rows, threads)
+    per_frame = float(np.mean([run.frame() for _ in range(frames)]))
+    return {"value": 1.0 / per_frame, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": run.sample(frames),
+            "measured_seconds": run.measured, "ms_per_frame_extrapolated": per_frame * 1e3}
 
 
 def host_cores() -> int:
@@ -186,17 +198,17 @@ def run_reference(args) -> None:
         return
     cfg = workload_config()
     threads = host_cores()
-    # one bounded sample per step
+    # one bounded sample (a frame with attention on sampled rows) per step; the whole run is bounded in time
+    run = OracleRunner(cfg, args.ref_rows, threads)
     per = []
-    total = args.warmup + args.steps
-    res = None
     t0 = time.perf_counter()
-    for i in range(total):
-        res = oracle_rate(cfg, frames=1, attn_rows=args.ref_rows, threads=threads)
+    for i in range(args.warmup + args.steps):
+        sec = run.frame()
         if i >= args.warmup:
-            per.append(res["ms_per_frame_extrapolated"])
-        if time.perf_counter() - t0 > 240 and i >= args.warmup:
+            per.append(sec * 1e3)
+        if time.perf_counter() - t0 > 120 and i >= args.warmup:
             break
+    res = {"sample": run.sample(len(per)) + ("; stopped after 120 s" if len(per) < args.steps else "")}
     ms = float(np.mean(per))
     value = 1e3 / ms
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
@@ -371,14 +383,14 @@ def run_ours(args) -> None:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=10000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--pool", type=int, default=160, help="distinct frames kept on the device (cycled beyond)")
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--profile-steps", type=int, default=100)
-    ap.add_argument("--cpu-frames", type=int, default=2)
-    ap.add_argument("--ref-rows", type=int, default=64)
+    ap.add_argument("--cpu-frames", type=int, default=8)
+    ap.add_argument("--ref-rows", type=int, default=96)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
