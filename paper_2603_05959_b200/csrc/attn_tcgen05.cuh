@@ -1,25 +1,18 @@
 // bf16 flash attention for sm_100a: out = softmax(Q K^T / sqrt(64)) V per head, head_dim 64, no mask.
 //
-// One CTA (one per SM) owns one 128-row query tile of one head and a contiguous range of 128-row KV tiles.
-// Tensor memory holds S_0, S_1 (fp32 scores of two KV tiles in flight), P_0, P_1 (bf16 probabilities) and O, so
-// every stage has its own buffer and the MMAs run ahead of the softmax:
-//   warps 0-3   softmax of the even KV tiles, warps 4-7 of the odd ones.  Thread (warp w, lane) owns query row
-//               32 (w mod 4) + lane: it reads its 128 scores with tcgen05.ld and releases the S buffer at once,
-//               hands the row maximum to the thread that owns the same row in the other warpgroup (shared
-//               memory, one mbarrier per direction and pair of warps) so that both replay the same sequence of
-//               reference maxima (O is rescaled, by the thread whose tile raised the maximum by more than 2^8,
-//               between the two P V products concerned), writes P as bf16, and at the end normalises and
-//               stores 32 columns of O
-//   warp 8      TMA producer: Q once, then K and V tiles into 128-byte-swizzled shared-memory stages
-//   warp 9      allocates tensor memory; issues S_b = Q K^T  (tcgen05.mma, both operands in shared memory)
-//   warp 10     issues O += P_b V (P read from tensor memory as the A operand, V MN-major from shared memory)
-// What shaped this: (1) one thread issues at most one tcgen05.mma per ~60 cycles and a commit costs about as
-// much, so with a single issuer the MMA loop alone (no softmax work at all) takes three quarters of the
-// kernel's time: hence two issuers and 128-column score MMAs; (2) every barrier round of a softmax warp costs
-// about a thousand cycles of latency (tensor-memory loads and stores, fences, mbarrier round trips, the
-// maximum's dependency chain) whatever the number of elements: hence 128 columns per round; (3) with head_dim
-// 64 a 128 x 128 tile needs 512 tensor-pipe cycles but 1024 cycles of the 16-per-clock exponential unit, so
-// two softmax warps per scheduler, alternating, are needed to keep that unit busy.  The KV range may be split
+// One CTA owns one 128-row query tile of one head and a contiguous range of 128-row KV tiles.  Each KV
+// tile is processed as two 64-row halves with their own S buffer in tensor memory, so the MMAs of one half
+// run while the softmax warps work on the other and the softmax never waits for a whole QK^T -> PV chain.
+//   warps 0-3   softmax: one thread per query row reads its 64 S values of a half with tcgen05.ld, keeps a
+//               running reference maximum (rescaling O only when the maximum grows by more than 2^8),
+//               writes P as bf16 over the first 32 columns of that half, and at the end normalises and stores O
+//   warp 4      TMA producer: Q once, then K and V tiles into 128-byte-swizzled shared-memory stages
+//   warp 5      allocates tensor memory and issues tcgen05.mma:  S_h = Q K_h^T  (SS, fp32 in TMEM),
+//               O += P_h V_h (P read from TMEM as the A operand, V MN-major from shared memory)
+//   warps 6-7   only complete the second warpgroup, which hands its registers to the softmax warpgroup
+// With head_dim 64 a 128 x 128 tile needs 512 tensor-pipe cycles but 1024 cycles of the 16-per-clock
+// exponential unit, so the exponentials bound the kernel; two CTAs are resident per SM (256 TMEM columns and
+// ~82 KB shared memory each) to keep that unit fed from two independent query tiles.  The KV range may be split
 // across CTAs; partial (O, max, sum) triples are merged by a second kernel.  Every mbarrier wait is bounded: on
 // expiry the CTA records OVGGT_ERR_TIMEOUT in the status word and leaves through the common teardown.
 #pragma once
@@ -33,25 +26,19 @@ namespace ovggt {
 constexpr int kBM = 128;            // query rows per CTA
 constexpr int kBN = 128;            // KV rows per tile
 constexpr int kHD = 64;             // head dim
-constexpr int kKVStages = 3;
-constexpr int kAttnThreads = 384;
-// 384 x 168 = 256 x 216 + 128 x 72 registers: the softmax warps' raise is exactly what the third warpgroup releases.
-constexpr int kRegsSoftmax = 216, kRegsOther = 72;
+constexpr int kKVStages = 2;
+constexpr int kAttnThreads = 256;
+constexpr int kRegsSoftmax = 216, kRegsOther = 40;   // 2 CTAs x (128 x 216 + 128 x 40) = 64K registers
 constexpr int kTileBytes = kBN * kHD * 2;          // 16 KB
 constexpr int kHalf = kBN / 2;      // KV rows per S buffer
-constexpr int kTmemCols = 512;
-constexpr int kColS = 0, kColP = 256, kColO = 384;   // S_b: 128 columns each; P_b: 64 columns each; O: 64 columns
+constexpr int kTmemCols = 256;
+constexpr int kColS = 0, kColO = 128;   // S_0 at columns [0, 64), S_1 at [64, 128), O at [128, 192)
 constexpr float kRescaleThreshold = 8.0f;          // log2 units
 constexpr int kMaxSplits = 16;
 
 struct AttnBarriers {
-  unsigned long long q_full, o_full, drain[2];
-  unsigned long long k_full[kKVStages], k_empty[kKVStages], v_full[kKVStages], v_empty[kKVStages];
-  unsigned long long s_full[2], s_free[2], p_full[2], pv_done[2];
-  unsigned long long pub[2][4];    // [warpgroup][quarter]: that warp has handed over the row maxima of its next tile
-  unsigned long long pair[4];      // rendezvous of the two warps that share query rows [32 q, 32 q + 32)
-  float xmx[2][2][kBM];            // [warpgroup][parity of its tile count][row]: row maximum of the tile (log2 units)
-  float xl[2][kBM];                // [warpgroup][row]: row sums, exchanged at the end
+  unsigned long long q_full, s_full[2], p_full[2], pv_done, o_full, drain;
+  unsigned long long k_full[kKVStages], v_full[kKVStages];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -173,22 +160,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
       "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -236,7 +207,7 @@ struct AttnParams {
   int* status;
 };
 
-__global__ void __launch_bounds__(kAttnThreads, 1)
+__global__ void __launch_bounds__(kAttnThreads, 2)
 k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const AttnParams P) {
   extern __shared__ unsigned char smem_raw[];
@@ -254,31 +225,22 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
   if (threadIdx.x == 0) {
     mbar_init(&B->q_full, 1);
-    mbar_init(&B->o_full, 1);
-    mbar_init(&B->drain[0], 1);
-    mbar_init(&B->drain[1], 1);
-    for (int s = 0; s < kKVStages; ++s) {
-      mbar_init(&B->k_full[s], 1);
-      mbar_init(&B->k_empty[s], 1);
-      mbar_init(&B->v_full[s], 1);
-      mbar_init(&B->v_empty[s], 1);
-    }
     for (int hf = 0; hf < 2; ++hf) {
       mbar_init(&B->s_full[hf], 1);
-      mbar_init(&B->s_free[hf], 4);      // one arrival per softmax warp of the half
-      mbar_init(&B->p_full[hf], 4);
-      mbar_init(&B->pv_done[hf], 1);
+      mbar_init(&B->p_full[hf], 128);
     }
-    for (int q = 0; q < 4; ++q) {
-      mbar_init(&B->pair[q], 2);
-      mbar_init(&B->pub[0][q], 1);
-      mbar_init(&B->pub[1][q], 1);
+    mbar_init(&B->pv_done, 1);
+    mbar_init(&B->o_full, 1);
+    mbar_init(&B->drain, 1);
+    for (int s = 0; s < kKVStages; ++s) {
+      mbar_init(&B->k_full[s], 1);
+      mbar_init(&B->v_full[s], 1);
     }
     B->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 9) {
+  if (warp == 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&B->tmem_base)),
                  "r"((uint32_t)kTmemCols)
                  : "memory");
@@ -289,9 +251,9 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem = *(volatile uint32_t*)&B->tmem_base;
 
-  if (warp >= 8) {
+  if (warp >= 4) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
-  if (warp == 8) {
+  if (warp == 4) {
     // ------------------------------------------------ TMA producer
     if (lane == 0) {
       int issued_k = 0, issued_v = 0;
@@ -302,12 +264,16 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int s = it % kKVStages;
         const uint32_t ph = (uint32_t)(it / kKVStages) & 1u;
         const int row = (t_begin + it) * kBN;
-        ok = mbar_wait(&B->k_empty[s], ph ^ 1u, B, P.status);
+        // stage s last held the keys of tile it - 2: free once both score MMAs of that tile have completed, which
+        // is what the completion of s_full[1] for that tile says (a commit covers every earlier MMA of the thread)
+        if (it >= kKVStages) ok = mbar_wait(&B->s_full[1], (uint32_t)(it - kKVStages) & 1u, B, P.status);
         if (!ok) break;
         mbar_expect_tx(&B->k_full[s], kTileBytes);
         tma_load_2d(sK + s * kTileBytes, &tm_k, h * kHD, row, &B->k_full[s]);
         ++issued_k;
-        ok = mbar_wait(&B->v_empty[s], ph ^ 1u, B, P.status);
+        // ... and the values of tile it - 2: their last reader, P V of its second half, is issued before the second
+        // score MMA of tile it - 1, so s_full[1] of tile it - 1 covers it
+        if (it >= kKVStages) ok = mbar_wait(&B->s_full[1], (uint32_t)(it - kKVStages + 1) & 1u, B, P.status);
         if (!ok) break;
         mbar_expect_tx(&B->v_full[s], kTileBytes);
         tma_load_2d(sV + s * kTileBytes, &tm_v, h * kHD, row, &B->v_full[s]);
@@ -322,134 +288,113 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           mbar_wait(&B->v_full[i % kKVStages], (uint32_t)(i / kKVStages) & 1u, B, P.status);
       }
     }
-  } else if (warp == 9) {
-    // ------------------------------------------------ issuer of S_b = Q K^T, b = tile parity
+    __syncwarp();
+  } else if (warp == 5) {
+    // ------------------------------------------------ MMA issuer
+    // Issue order (the tensor pipe executes one thread's MMAs in order):
+    //   QK(0,0) QK(0,1) | PV(0,0) QK(1,0) PV(0,1) QK(1,1) | PV(1,0) QK(2,0) PV(1,1) QK(2,1) | ...
+    // QK(t+1,h) overwrites S_h only after PV(t,h) has read P_h from it.
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = idesc_bf16(kBN, false);
+      constexpr uint32_t idesc_qk = idesc_bf16(kHalf, false);
+      constexpr uint32_t idesc_pv = idesc_bf16(kHD, true);
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ));
-      bool ok = mbar_wait(&B->q_full, 0, B, P.status);
-      for (int it = 0; it < n_tiles && ok; ++it) {
-        const int s = it % kKVStages, b = it & 1;
-        ok = mbar_wait(&B->k_full[s], (uint32_t)(it / kKVStages) & 1u, B, P.status);
-        // the softmax warps must have read the previous content of S_b (tile it - 2)
-        if (ok && it >= 2) ok = mbar_wait(&B->s_free[b], (uint32_t)((it >> 1) - 1) & 1u, B, P.status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint64_t dk = smem_desc_sw128(smem_u32(sK + s * kTileBytes));
+      // S_hf = Q K_hf^T for the KV tile held in stage `st` (64 rows = 8 swizzle groups = 8192 bytes per half)
+      auto issue_qk = [&](int st, int hf) {
+        const uint64_t dk = smem_desc_sw128(smem_u32(sK + st * kTileBytes + hf * (kTileBytes / 2)));
 #pragma unroll
         for (int kk = 0; kk < kHD / 16; ++kk)     // 16 elements of head dim = 32 bytes inside the swizzled row
-          mma_ss(tmem + kColS + b * kBN, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_qk, kk > 0);
-        tc_commit(&B->s_full[b]);
-        tc_commit(&B->k_empty[s]);
-      }
-      if (!ok) {
-        tc_commit(&B->drain[0]);                    // let every issued MMA finish before TMEM is freed
-        mbar_wait(&B->drain[0], 0, B, P.status);
-      }
-    }
-  } else if (warp == 10) {
-    // ------------------------------------------------ issuer of O += P_b V
-    if (lane == 0) {
-      constexpr uint32_t idesc_pv = idesc_bf16(kHD, true);
-      bool ok = true;
-      for (int it = 0; it < n_tiles && ok; ++it) {
-        const int s = it % kKVStages, b = it & 1;
-        ok = mbar_wait(&B->v_full[s], (uint32_t)(it / kKVStages) & 1u, B, P.status);
-        if (ok) ok = mbar_wait(&B->p_full[b], (uint32_t)(it >> 1) & 1u, B, P.status);
-        if (!ok) break;
+          mma_ss(tmem + kColS + hf * kHalf, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_qk, kk > 0);
+      };
+      bool ok = mbar_wait(&B->q_full, 0, B, P.status);
+      if (ok) ok = mbar_wait(&B->k_full[0], 0, B, P.status);
+      if (ok) {
         tc_fence_after();
+        issue_qk(0, 0);
+        tc_commit(&B->s_full[0]);
+        issue_qk(0, 1);
+        tc_commit(&B->s_full[1]);
+      }
+      for (int it = 0; it < n_tiles && ok; ++it) {
+        const int s = it % kKVStages, s1 = (it + 1) % kKVStages;
+        const uint32_t ph = (uint32_t)(it / kKVStages) & 1u, ph1 = (uint32_t)((it + 1) / kKVStages) & 1u;
+        const bool more = it + 1 < n_tiles;
+        ok = mbar_wait(&B->v_full[s], ph, B, P.status);
+        if (!ok) break;
         const uint64_t dv = smem_desc_sw128(smem_u32(sV + s * kTileBytes));
 #pragma unroll
-        for (int kk = 0; kk < kBN / 16; ++kk)       // 16 KV rows = 2048 bytes; P: 8 TMEM columns per 16 bf16
-          mma_ts(tmem + kColO, tmem + kColP + b * (kBN / 2) + kk * 8, dv + (uint64_t)(kk * 128), idesc_pv,
-                 (it > 0 || kk > 0));
-        tc_commit(&B->pv_done[b]);
-        tc_commit(&B->v_empty[s]);
+        for (int hf = 0; hf < 2; ++hf) {
+          ok = mbar_wait(&B->p_full[hf], (uint32_t)it & 1u, B, P.status);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = 0; kk < kHalf / 16; ++kk)   // 16 KV rows = 2048 bytes; P: 8 TMEM columns per 16 bf16
+            mma_ts(tmem + kColO, tmem + kColS + hf * kHalf + kk * 8, dv + (uint64_t)((hf * (kHalf / 16) + kk) * 128),
+                   idesc_pv, (it > 0 || hf > 0 || kk > 0));
+          if (!more && hf == 0) tc_commit(&B->pv_done);   // (the last half has no later score MMA to tell it by)
+          if (more) {
+            if (hf == 0) {
+              ok = mbar_wait(&B->k_full[s1], ph1, B, P.status);
+              if (!ok) break;
+              tc_fence_after();
+            }
+            issue_qk(s1, hf);
+            tc_commit(&B->s_full[hf]);
+          }
+        }
       }
       if (ok) {
         tc_commit(&B->o_full);
+        mbar_wait(&B->o_full, 0, B, P.status);
       } else {
-        tc_commit(&B->drain[1]);
-        mbar_wait(&B->drain[1], 0, B, P.status);
+        tc_commit(&B->drain);                     // let every issued MMA finish before TMEM is freed
+        mbar_wait(&B->drain, 0, B, P.status);
       }
     }
+    __syncwarp();
   }
-  __syncwarp();
   } else {
-    // ------------------------------------------------ softmax, correction and epilogue (8 warps)
+    // ------------------------------------------------ softmax, correction and epilogue (128 threads)
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-    const int wg = warp >> 2, quad = warp & 3;         // parity of this warpgroup's tiles, lane quarter of tensor memory
+    const int quad = warp;
     const int row = quad * 32 + lane;
     const uint32_t t_row = tmem + ((uint32_t)(quad * 32) << 16);
     const float c = 1.4426950408889634f * 0.125f;     // log2(e) / sqrt(64)
-    // mref: reference maximum of the row after the last tile either thread of the row has accounted for;
-    // l: sum of this thread's own P values, in units of 2^mref
     float mref = 0.0f, l = 0.0f;
     bool ok = true;
-    // the other thread's tile raised the maximum: follow it (that thread rescales O)
-    auto follow = [&](float m) {
-      if (m - mref > kRescaleThreshold) {
-        l *= ex2(mref - m);
-        mref = m;
-      }
-    };
-    for (int it = wg; it < n_tiles; it += 2) {
-      const int k = it >> 1;                            // this warpgroup's k-th tile: phase of its per-buffer barriers
-      ok = mbar_wait(&B->s_full[wg], (uint32_t)k & 1u, B, P.status);
+    for (int idx = 0; idx < 2 * n_tiles; ++idx) {       // idx = 2 * tile + half
+      const int it = idx >> 1, hf = idx & 1;
+      ok = mbar_wait(&B->s_full[hf], (uint32_t)it & 1u, B, P.status);
       if (!ok) break;
       tc_fence_after();
-      uint32_t s[kBN];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) tmem_ld32(t_row + kColS + wg * kBN + j * 32, s + j * 32);
+      uint32_t s[kHalf];
+      tmem_ld32(t_row + kColS + hf * kHalf, s);
+      tmem_ld32(t_row + kColS + hf * kHalf + 32, s + 32);
       tmem_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&B->s_free[wg]);       // S_b may be overwritten by the scores of tile it + 2
-      const int col0 = (t_begin + it) * kBN;
-      if (col0 + kBN > P.N) {
+      const int col0 = (t_begin + it) * kBN + hf * kHalf;
+      if (col0 + kHalf > P.N) {
 #pragma unroll
-        for (int j = 0; j < kBN; ++j)
-          if (col0 + j >= P.N) s[j] = 0xFF800000u;       // -inf on columns past the last row
+        for (int j = 0; j < kHalf; ++j)
+          if (col0 + j >= P.N) s[j] = 0xFF800000u;     // -inf on columns past the last row
       }
-      // row maximum: eight independent chains of 3-input maxima
-      float mx;
-      {
-        float m8[8];
+      // row maximum: four independent chains of 3-input maxima
+      float m4[4];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          m8[q] = fmaxf(__uint_as_float(s[16 * q]), __uint_as_float(s[16 * q + 1]));
+      for (int q = 0; q < 4; ++q) {
+        m4[q] = fmaxf(__uint_as_float(s[16 * q]), __uint_as_float(s[16 * q + 1]));
 #pragma unroll
-          for (int j = 2; j < 16; j += 2)
-            m8[q] = max3(m8[q], __uint_as_float(s[16 * q + j]), __uint_as_float(s[16 * q + j + 1]));
-        }
-        mx = max3(max3(m8[0], m8[1], m8[2]), max3(m8[3], m8[4], m8[5]), fmaxf(m8[6], m8[7])) * c;
+        for (int j = 2; j < 16; j += 2)
+          m4[q] = max3(m4[q], __uint_as_float(s[16 * q + j]), __uint_as_float(s[16 * q + j + 1]));
       }
-      // The tiles of a row are accounted for in order.  Take the maximum of the tile before this one from the other
-      // thread, then hand over this one's.  (Waiting before handing over keeps the two barriers of a pair strictly
-      // alternating, so a parity wait cannot alias.)
-      if (it > 0) {
-        // tile it - 1 is the other warpgroup's tile number (it - 1) >> 1
-        const int kp = (it - 1) >> 1;
-        ok = mbar_wait(&B->pub[wg ^ 1][quad], (uint32_t)kp & 1u, B, P.status);
-        if (!ok) break;
-        const float m_prev = B->xmx[wg ^ 1][kp & 1][row];
-        if (it == 1) mref = m_prev; else follow(m_prev);
-      }
-      B->xmx[wg][k & 1][row] = mx;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&B->pub[wg][quad]);
-      // This warpgroup's P buffer is free once the P V of its previous tile (it - 2) has completed.  Waiting here,
-      // every tile, also keeps the parity wait of the rescaling path below unambiguous: the P V products complete
-      // in issue order, so the other buffer's barrier is then at most one phase behind the one waited for.
-      if (it >= 2) ok = mbar_wait(&B->pv_done[wg], (uint32_t)(k - 1) & 1u, B, P.status);
-      if (!ok) break;
-      if (it == 0) {
+      float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * c;
+      if (idx == 0) {
         mref = mx;
       } else {
         const bool grow = mx - mref > kRescaleThreshold;
         if (__any_sync(0xFFFFFFFFu, grow)) {
-          // O must hold every earlier tile and nothing else: wait for the P V of tile it - 1
-          ok = mbar_wait(&B->pv_done[wg ^ 1], (uint32_t)((it - 1) >> 1) & 1u, B, P.status);
+          // O may still be accumulating the previous half.  PV(idx - 1) is issued just before the scores of half
+          // idx + 1, so the completion of those scores covers it; the last half has a barrier of its own.
+          ok = idx + 1 < 2 * n_tiles ? mbar_wait(&B->s_full[hf ^ 1], (uint32_t)((idx + 1) >> 1) & 1u, B, P.status)
+                                     : mbar_wait(&B->pv_done, 0, B, P.status);
           if (!ok) break;
           tc_fence_after();
           const float a = grow ? ex2(mref - mx) : 1.0f;
@@ -457,16 +402,15 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             mref = mx;
             l *= a;
           }
-#pragma unroll 1
-          for (int j = 0; j < 4; ++j) {                   // (rare path: keep its register use small)
-            uint32_t o[16];
-            tmem_ld16(t_row + kColO + j * 16, o);
+          uint32_t o[32];
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            tmem_ld32(t_row + kColO + j * 32, o);
             tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * a);
-            tmem_st16(t_row + kColO + j * 16, o);
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * a);
+            tmem_st32(t_row + kColO + j * 32, o);
           }
-          tmem_wait_st();
         }
       }
       // p = 2^(s * c - mref) on pairs; four independent packed partial sums, folded in a fixed order
@@ -475,7 +419,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
       for (int q = 0; q < 4; ++q) acc[q] = make_float2(0.0f, 0.0f);
 #pragma unroll
-      for (int j = 0; j < kBN; j += 2) {
+      for (int j = 0; j < kHalf; j += 2) {
         const float2 x = fma2(make_float2(__uint_as_float(s[j]), __uint_as_float(s[j + 1])), c2, nm2);
         const float2 p = make_float2(ex2(x.x), ex2(x.y));
         acc[(j >> 1) & 3] = add2(acc[(j >> 1) & 3], p);
@@ -483,65 +427,48 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       const float2 t = add2(add2(acc[0], acc[1]), add2(acc[2], acc[3]));
       l += t.x + t.y;
-      tmem_st32(t_row + kColP + wg * (kBN / 2), s);
-      tmem_st32(t_row + kColP + wg * (kBN / 2) + 32, s + 32);
+      tmem_st32(t_row + kColS + hf * kHalf, s);
       tmem_wait_st();
       tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&B->p_full[wg]);
-    }
-    // the warpgroup that did not have the last tile follows it
-    if (ok && ((n_tiles - 1) & 1) != wg) {
-      const int kp = (n_tiles - 1) >> 1;
-      ok = mbar_wait(&B->pub[wg ^ 1][quad], (uint32_t)kp & 1u, B, P.status);
-      if (ok) {
-        const float m_last = B->xmx[wg ^ 1][kp & 1][row];
-        if (n_tiles == 1) mref = m_last; else follow(m_last);   // (a single tile: this warpgroup had none)
-      }
-    }
-    // row sum over both warpgroups
-    float l_all = l;
-    if (ok) {
-      B->xl[wg][row] = l;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&B->pair[quad]);
-      ok = mbar_wait(&B->pair[quad], 0, B, P.status);
-      if (ok) l_all = B->xl[0][row] + B->xl[1][row];
+      mbar_arrive(&B->p_full[hf]);
     }
     if (ok) ok = mbar_wait(&B->o_full, 0, B, P.status);
     if (ok) {
       tc_fence_after();
       const int m = qt * kBM + row;
-      const float inv = 1.0f / l_all;
-      uint32_t o[32];                                     // this thread's share: columns [32 wg, 32 wg + 32) of the row
-      tmem_ld32(t_row + kColO + wg * 32, o);
-      tmem_wait_ld();
-      if (m < P.M) {
-        if (P.splits == 1) {
-          uint4* dst = reinterpret_cast<uint4*>(P.out + (size_t)m * C + (size_t)h * kHD + wg * 32);
+      const float inv = 1.0f / l;
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            uint4 w;
-            w.x = pack_bf16(__uint_as_float(o[8 * e + 0]) * inv, __uint_as_float(o[8 * e + 1]) * inv);
-            w.y = pack_bf16(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv);
-            w.z = pack_bf16(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv);
-            w.w = pack_bf16(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv);
-            dst[e] = w;
+      for (int j = 0; j < 2; ++j) {
+        uint32_t o[32];
+        tmem_ld32(t_row + kColO + j * 32, o);
+        tmem_wait_ld();
+        if (m < P.M) {
+          if (P.splits == 1) {
+            uint4* dst = reinterpret_cast<uint4*>(P.out + (size_t)m * C + (size_t)h * kHD + j * 32);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              uint4 w;
+              w.x = pack_bf16(__uint_as_float(o[8 * e + 0]) * inv, __uint_as_float(o[8 * e + 1]) * inv);
+              w.y = pack_bf16(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv);
+              w.z = pack_bf16(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv);
+              w.w = pack_bf16(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv);
+              dst[e] = w;
+            }
+          } else {
+            uint4* dst = reinterpret_cast<uint4*>(P.o_part + ((size_t)split * P.M + m) * C + (size_t)h * kHD + j * 32);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) dst[e] = make_uint4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
           }
-        } else {
-          uint4* dst = reinterpret_cast<uint4*>(P.o_part + ((size_t)split * P.M + m) * C + (size_t)h * kHD + wg * 32);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) dst[e] = make_uint4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
-          if (wg == 0) P.ml_part[((size_t)split * P.M + m) * P.H + h] = make_float2(mref, l_all);
         }
       }
+      if (P.splits > 1 && m < P.M) P.ml_part[((size_t)split * P.M + m) * P.H + h] = make_float2(mref, l);
     }
   }
 
   // ------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) {
+  if (warp == 5) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols) : "memory");
   }
@@ -615,10 +542,10 @@ inline int make_rows_map(CUtensorMap* map, const void* base, int rows, int C) {
   return OVGGT_OK;
 }
 
-// Number of KV splits: minimise (waves of CTAs over 148 slots, one per SM) x (tiles per CTA + fixed overhead).
+// Number of KV splits: minimise (waves of CTAs over 2 x 148 slots) x (tiles per CTA + fixed overhead).
 inline int attn_choose_splits(int M, int N, int H) {
   const int q_tiles = (M + kBM - 1) / kBM, tiles = (N + kBN - 1) / kBN;
-  const long slots = 148;
+  const long slots = 2L * 148;
   int best = 1;
   long best_cost = -1;
   for (int s = 1; s <= kMaxSplits && s <= tiles; ++s) {
