@@ -474,7 +474,8 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   }
 }
 
-// out[m, h*64 + c] = sum_s O_s 2^(m_s - m*) / sum_s l_s 2^(m_s - m*), m* = max_s m_s.  One thread per 4 columns.
+// out[m, h*64 + c] = sum_s O_s 2^(m_s - m*) / sum_s l_s 2^(m_s - m*), m* = max_s m_s, splits folded in order.
+// One thread per 4 columns; all loads of a thread are issued before the arithmetic that needs them.
 __global__ void __launch_bounds__(256) k_attn_merge(const float* __restrict__ o_part, const float2* __restrict__ ml_part,
                                                     int M, int H, int splits, __nv_bfloat16* __restrict__ out) {
   const int C = H * kHD;
@@ -482,20 +483,30 @@ __global__ void __launch_bounds__(256) k_attn_merge(const float* __restrict__ o_
   const size_t total = (size_t)M * (C / 4);
   if (idx >= total) return;
   const int m = (int)(idx / (C / 4)), c4 = (int)(idx % (C / 4)), h = (c4 * 4) / kHD;
+  float2 ml[kMaxSplits];
+  float4 o[kMaxSplits];
+#pragma unroll
+  for (int s = 0; s < kMaxSplits; ++s)
+    if (s < splits) {
+      ml[s] = ml_part[((size_t)s * M + m) * H + h];
+      o[s] = *reinterpret_cast<const float4*>(o_part + ((size_t)s * M + m) * C + c4 * 4);
+    }
   float mstar = -INFINITY;
-  for (int s = 0; s < splits; ++s) mstar = fmaxf(mstar, ml_part[((size_t)s * M + m) * H + h].x);
+#pragma unroll
+  for (int s = 0; s < kMaxSplits; ++s)
+    if (s < splits) mstar = fmaxf(mstar, ml[s].x);
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   float den = 0.0f;
-  for (int s = 0; s < splits; ++s) {
-    const float2 ml = ml_part[((size_t)s * M + m) * H + h];
-    const float w = exp2f(ml.x - mstar);
-    const float4 o = *reinterpret_cast<const float4*>(o_part + ((size_t)s * M + m) * C + c4 * 4);
-    acc.x = fmaf(w, o.x, acc.x);
-    acc.y = fmaf(w, o.y, acc.y);
-    acc.z = fmaf(w, o.z, acc.z);
-    acc.w = fmaf(w, o.w, acc.w);
-    den = fmaf(w, ml.y, den);
-  }
+#pragma unroll
+  for (int s = 0; s < kMaxSplits; ++s)
+    if (s < splits) {
+      const float w = exp2f(ml[s].x - mstar);
+      acc.x = fmaf(w, o[s].x, acc.x);
+      acc.y = fmaf(w, o[s].y, acc.y);
+      acc.z = fmaf(w, o[s].z, acc.z);
+      acc.w = fmaf(w, o[s].w, acc.w);
+      den = fmaf(w, ml[s].y, den);
+    }
   const float inv = 1.0f / den;
   uint2 w;
   w.x = pack_bf16(acc.x * inv, acc.y * inv);

@@ -97,8 +97,10 @@ int launch_diversity(const void* K, int rows, int C, int dtype, float* part, flo
   LAUNCHED();
   const int grid = std::min((rows + 7) / 8, 148 * 8);
   const size_t smem = (size_t)C * 4;
-  if (dtype == kBF16) k_diversity<kBF16><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d);
-  else                k_diversity<kF32><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d);
+  if (dtype == kBF16)
+    k_diversity<kBF16><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d, grid, nullptr, 0, nullptr);
+  else
+    k_diversity<kF32><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d, grid, nullptr, 0, nullptr);
   LAUNCHED();
   return OVGGT_OK;
 }
@@ -107,16 +109,22 @@ constexpr int kColsumSlices = 8;
 
 // Diversity from the per-CTA column sums the last compaction left (nparts rows of part): no pass over K for the sums.
 // slices: [kColsumSlices, C] floats.
+// The same launch also computes the residual norms s_raw [resid_rows] of the new frame when resid is given.
 int launch_diversity_from_parts(const void* K, int rows, int C, int dtype, const float* part, int nparts, float* slices,
-                                float* d, cudaStream_t st) {
+                                float* d, const void* resid, int resid_rows, float* s_raw, cudaStream_t st) {
   if (rows <= 0) return OVGGT_OK;
   const int nvec = C * elem_bytes(dtype) / 16;
   k_colsum_final_sliced<<<dim3((C + 31) / 32, kColsumSlices), 1024, 0, st>>>(part, nparts, C, slices);
   LAUNCHED();
   const int grid = std::min((rows + 15) / 16, 148 * 8);
   const size_t smem = (size_t)C * 4;
-  if (dtype == kBF16) k_diversity<kBF16><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, slices, kColsumSlices, d);
-  else                k_diversity<kF32><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, slices, kColsumSlices, d);
+  const int norm_ctas = resid ? (resid_rows + 7) / 8 : 0;
+  if (dtype == kBF16)
+    k_diversity<kBF16><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, slices, kColsumSlices, d, grid,
+                                                            (const uint4*)resid, resid_rows, s_raw);
+  else
+    k_diversity<kF32><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, slices, kColsumSlices, d, grid,
+                                                           (const uint4*)resid, resid_rows, s_raw);
   LAUNCHED();
   return OVGGT_OK;
 }
@@ -463,15 +471,18 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
   }
   const bool first = (t == h->first_frame);
 
-  {
+  // With column sums left by the last compaction, the residual norms ride in the diversity launch.
+  const bool fused_scores = c.score_mode == OVGGT_SCORE_HYBRID && n > 0 && S.colsum_nparts > 0;
+  if (!fused_scores) {
     ProfScope ps(h, OVGGT_PROF_ROW_NORMS, st);
     rc = launch_row_norms(io->resid, M, C, c.dtype, S.s_raw, st);
   }
   if (rc) return rc;
   if (c.score_mode == OVGGT_SCORE_HYBRID && n > 0) {
     ProfScope ps(h, OVGGT_PROF_DIVERSITY, st);
-    if (S.colsum_nparts > 0)
-      rc = launch_diversity_from_parts(S.kbuf[b], n, C, c.dtype, S.colsum_part, S.colsum_nparts, h->ksum, S.d, st);
+    if (fused_scores)
+      rc = launch_diversity_from_parts(S.kbuf[b], n, C, c.dtype, S.colsum_part, S.colsum_nparts, h->ksum, S.d,
+                                       io->resid, M, S.s_raw, st);
     else
       rc = launch_diversity(S.kbuf[b], n, C, c.dtype, h->colsum_part, h->ksum, S.d, st);
     if (rc) return rc;

@@ -10,12 +10,9 @@ namespace ovggt {
 // s[row] = sqrt(sum_c x[row, c]^2); one warp per row.  Lane l owns vectors l, l+32, ... and
 // folds them in that order; lanes are combined by the fixed butterfly of warp_sum.
 template <int DT>
-__global__ void __launch_bounds__(256) k_row_norms(const uint4* __restrict__ x, int rows, int nvec,
-                                                   float* __restrict__ s) {
+__device__ __forceinline__ void warp_row_norm(const uint4* __restrict__ x, int row, int nvec, float* __restrict__ s) {
   constexpr int VEC = VecOf<DT>::n;
   const int lane = threadIdx.x & 31;
-  const int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5);
-  if (row >= rows) return;
   const uint4* p = x + (size_t)row * nvec;
   float acc = 0.0f;
   for (int v0 = lane; v0 < nvec; v0 += 128) {
@@ -34,6 +31,13 @@ __global__ void __launch_bounds__(256) k_row_norms(const uint4* __restrict__ x, 
   }
   acc = warp_sum(acc);
   if (lane == 0) s[row] = __fsqrt_rn(acc);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(256) k_row_norms(const uint4* __restrict__ x, int rows, int nvec,
+                                                   float* __restrict__ s) {
+  const int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5);
+  if (row < rows) warp_row_norm<DT>(x, row, nvec, s);
 }
 
 // Column sums of K [rows, C], stage 1: CTA p sums its contiguous chunk of rows, in row order,
@@ -122,8 +126,17 @@ __global__ void __launch_bounds__(1024) k_colsum_final_sliced(const float* __res
 template <int DT>
 __global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, int rows, int nvec,
                                                    const float* __restrict__ ksum, int n_slices,
-                                                   float* __restrict__ d) {
+                                                   float* __restrict__ d, int div_ctas,
+                                                   const uint4* __restrict__ resid, int resid_rows,
+                                                   float* __restrict__ s_raw) {
   constexpr int VEC = VecOf<DT>::n;
+  // CTAs past the first div_ctas carry a second, independent job in the same launch: the residual norms of
+  // Eq. 5 (one warp per row), so that a step pays one launch for both scores.
+  if ((int)blockIdx.x >= div_ctas) {
+    const int row = (int)((((int)blockIdx.x - div_ctas) * (unsigned)blockDim.x + threadIdx.x) >> 5);
+    if (row < resid_rows) warp_row_norm<DT>(resid, row, nvec, s_raw);
+    return;
+  }
   extern __shared__ float sh_ksum[];
   const int C = nvec * VEC;
   for (int c = threadIdx.x; c < C; c += blockDim.x) {   // ksum: [n_slices, C], folded in slice order
@@ -138,7 +151,7 @@ __global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, 
 #pragma unroll
     for (int e = 0; e < VEC; ++e) kn = __fmaf_rn(sh_ksum[v * VEC + e], sh_ksum[v * VEC + e], kn);
   kn = warp_sum(kn);
-  const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
+  const int warps_total = (int)((div_ctas * (unsigned)blockDim.x) >> 5);
   // two rows per iteration, so that eight 16-byte loads per lane are in flight
   for (int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5) * 2; row < rows;
        row += 2 * warps_total) {
