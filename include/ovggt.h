@@ -126,7 +126,10 @@ int ovggt_layer_attend(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* 
  * score_override. */
 int ovggt_layer_compress(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
 
-/* ovggt_layer_attend followed by ovggt_layer_compress: the whole hot path of one (frame, layer). */
+/* ovggt_layer_attend followed by ovggt_layer_compress: the whole hot path of one (frame, layer).  The scoring
+ * kernels, which depend on neither the append nor the attention, are enqueued on a second stream that the handle
+ * owns (a host object, created by ovggt_cache_create), forked from and joined back into `stream` with events: for
+ * the caller the call is still asynchronous and ordered on `stream` alone. */
 int ovggt_layer_step(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
 
 /* The same step with HOST tensors: q, k, v, resid, conf, out are host pointers (pinned memory

@@ -194,6 +194,7 @@ struct LayerState {
   int* n_keep_dev;
   float* colsum_part = nullptr;   // [148 * 8, C]: per-CTA column sums of the keys the last compaction wrote
   int colsum_nparts = 0;          // 0: not available (the next step sums the keys itself)
+  int64_t scores_frame = -1;      // frame whose s_raw and d were already enqueued on the side stream
   size_t kv_bytes = 0;
 };
 
@@ -217,6 +218,10 @@ struct ovggt_cache {
   float w_center = 0, w_edge = 0, w_corner = 0;
   cudaStream_t last_stream = nullptr;
   int max_rows = 0;
+  // ovggt_layer_step scores the cache (diversity, residual norms) on a second, higher-priority stream while the
+  // attention runs: the scores do not depend on the attention.  Host objects only; absent if creation failed.
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   // optional per-kernel-class timing (host-side CUDA events; no device memory)
   bool prof = false;
   struct ProfRec { int cls; cudaEvent_t a, b; };
@@ -386,6 +391,19 @@ extern "C" int ovggt_cache_create(const ovggt_config* cfg, ovggt_cache** out) {
   h->w_center = (float)(1.0 / z);
   h->w_edge = (float)(e1 / z);
   h->w_corner = (float)(e2 / z);
+  {
+    int lo = 0, hi = 0;
+    if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess ||
+        cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, hi) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+      if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+      if (h->side) cudaStreamDestroy(h->side);
+      h->side = nullptr;
+      h->ev_fork = h->ev_join = nullptr;
+      (void)cudaGetLastError();
+    }
+  }
   cudaError_t e = cudaMemset(h->status, 0, 64);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
@@ -401,6 +419,12 @@ extern "C" int ovggt_cache_destroy(ovggt_cache* h) {
   for (auto& r : h->prof_recs) {
     cudaEventDestroy(r.a);
     cudaEventDestroy(r.b);
+  }
+  if (h->side) {
+    cudaStreamSynchronize(h->side);
+    cudaStreamDestroy(h->side);
+    cudaEventDestroy(h->ev_fork);
+    cudaEventDestroy(h->ev_join);
   }
   delete h;
   return OVGGT_OK;
@@ -473,12 +497,16 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
 
   // With column sums left by the last compaction, the residual norms ride in the diversity launch.
   const bool fused_scores = c.score_mode == OVGGT_SCORE_HYBRID && n > 0 && S.colsum_nparts > 0;
-  if (!fused_scores) {
+  const bool prelaunched = S.scores_frame == t;    // ovggt_layer_step already enqueued them on the side stream
+  S.scores_frame = -1;
+  if (prelaunched) {
+    CK(cudaStreamWaitEvent(st, h->ev_join, 0));
+  } else if (!fused_scores) {
     ProfScope ps(h, OVGGT_PROF_ROW_NORMS, st);
     rc = launch_row_norms(io->resid, M, C, c.dtype, S.s_raw, st);
   }
   if (rc) return rc;
-  if (c.score_mode == OVGGT_SCORE_HYBRID && n > 0) {
+  if (c.score_mode == OVGGT_SCORE_HYBRID && n > 0 && !prelaunched) {
     ProfScope ps(h, OVGGT_PROF_DIVERSITY, st);
     if (fused_scores)
       rc = launch_diversity_from_parts(S.kbuf[b], n, C, c.dtype, S.colsum_part, S.colsum_nparts, h->ksum, S.d,
@@ -539,8 +567,41 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
 }
 
 extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
-  int rc = ovggt_layer_attend(h, layer, io, stream);
+  int rc = check_layer(h, layer);
   if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The scores of the cached rows (key diversity) and of the new rows (residual norms) depend on neither the
+  // append nor the attention of this step: start them now on the side stream, join before the selection.
+  bool pre = false;
+  if (h->side && io && io->resid && aligned16(io->resid) && io->q && io->k && io->v && io->out) {
+    LayerState& S = h->layers[layer];
+    const ovggt_config& c = h->cfg;
+    if (!S.pending && c.score_mode == OVGGT_SCORE_HYBRID && S.n > 0 && S.colsum_nparts > 0 &&
+        io->frame_id > S.pending_frame) {
+      CK(cudaEventRecord(h->ev_fork, st));
+      CK(cudaStreamWaitEvent(h->side, h->ev_fork, 0));
+      {
+        ProfScope ps(h, OVGGT_PROF_DIVERSITY, h->side);
+        rc = launch_diversity_from_parts(S.kbuf[S.cur], S.n, h->C, c.dtype, S.colsum_part, S.colsum_nparts, h->ksum,
+                                         S.d, io->resid, h->M, S.s_raw, h->side);
+      }
+      CK(cudaEventRecord(h->ev_join, h->side));
+      if (rc) {
+        (void)cudaStreamWaitEvent(st, h->ev_join, 0);
+        return rc;
+      }
+      S.scores_frame = io->frame_id;
+      pre = true;
+    }
+  }
+  rc = ovggt_layer_attend(h, layer, io, stream);
+  if (rc) {
+    if (pre) {                          // keep the caller's stream ordered after the side work
+      (void)cudaStreamWaitEvent(st, h->ev_join, 0);
+      h->layers[layer].scores_frame = -1;
+    }
+    return rc;
+  }
   return ovggt_layer_compress(h, layer, io, stream);
 }
 
