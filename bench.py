@@ -307,11 +307,13 @@ def run_ours(args) -> None:
     per_step = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(K)])
 
     # ---- per-kernel device time (events around each kernel class; separate pass, same stream of frames)
+    cache.set_overlap(False)           # one kernel class at a time: the two halves of a step on one stream
     cache.profile_enable(True)
     for _ in range(n_prof):
         step(t_id); t_id += 1
     prof = cache.profile_read(reset=True)
     cache.profile_enable(False)
+    cache.set_overlap(True)
     clocks = sampler.stop()
 
     # ---- end to end: host buffers through the C ABI, copies inside the timed region

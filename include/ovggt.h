@@ -126,11 +126,15 @@ int ovggt_layer_attend(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* 
  * score_override. */
 int ovggt_layer_compress(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
 
-/* ovggt_layer_attend followed by ovggt_layer_compress: the whole hot path of one (frame, layer).  The scoring
- * kernels, which depend on neither the append nor the attention, are enqueued on a second stream that the handle
- * owns (a host object, created by ovggt_cache_create), forked from and joined back into `stream` with events: for
- * the caller the call is still asynchronous and ordered on `stream` alone. */
+/* ovggt_layer_attend and ovggt_layer_compress of one (frame, layer): the whole hot path.  The compress half reads
+ * the cache and the new rows but not the attention's output, so it is enqueued on a second stream that the handle
+ * owns (a host object, created by ovggt_cache_create), forked from and joined back into `stream` with events, and
+ * runs beside the attention.  For the caller the call is still asynchronous and ordered on `stream` alone. */
 int ovggt_layer_step(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
+
+/* Turn the overlap of ovggt_layer_step off (0) or on (non-zero, the default): off, the two halves run one after the
+ * other on `stream`, which is what per-kernel timing wants. */
+int ovggt_cache_set_overlap(ovggt_cache* cache, int32_t enable);
 
 /* The same step with HOST tensors: q, k, v, resid, conf, out are host pointers (pinned memory
  * makes the copies asynchronous); score_override must be NULL.  The inputs are copied into staging

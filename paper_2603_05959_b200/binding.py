@@ -25,7 +25,7 @@ EXPORTED = [
     "ovggt_workspace_bytes", "ovggt_cache_create", "ovggt_cache_destroy", "ovggt_layer_attend",
     "ovggt_layer_compress", "ovggt_layer_step", "ovggt_layer_step_host", "ovggt_cache_stats",
     "ovggt_cache_export", "ovggt_cache_import", "ovggt_cache_last_selection", "ovggt_kernel_launches",
-    "ovggt_cache_profile_enable", "ovggt_cache_profile_read",
+    "ovggt_cache_profile_enable", "ovggt_cache_profile_read", "ovggt_cache_set_overlap",
     "ovggt_strerror", "ovggt_last_cuda_error", "ovggt_k_row_norms", "ovggt_k_diversity_scratch_bytes",
     "ovggt_k_diversity", "ovggt_k_diversity_static", "ovggt_k_select", "ovggt_k_compact", "ovggt_k_attention_scratch_bytes",
     "ovggt_k_attention",
@@ -93,6 +93,7 @@ def lib():
         L.ovggt_cache_import.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32, i64, i64]
         L.ovggt_cache_last_selection.argtypes = [vp, i32, vp, C.POINTER(i32), vp, C.POINTER(i32)]
         L.ovggt_cache_profile_enable.argtypes = [vp, i32]
+        L.ovggt_cache_set_overlap.argtypes = [vp, i32]
         L.ovggt_cache_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), i32]
         L.ovggt_kernel_launches.restype = C.c_uint64
         L.ovggt_strerror.restype = C.c_char_p
@@ -258,6 +259,9 @@ class OvggtCache:
         _check(lib().ovggt_cache_import(self._h, layer, ids.ctypes.data, flags.ctypes.data, scores.ctypes.data,
                                         k.ctypes.data, v.ctypes.data, len(ids), int(next_frame_id),
                                         int(last_registration_frame)), "ovggt_cache_import")
+
+    def set_overlap(self, on: bool) -> None:
+        _check(lib().ovggt_cache_set_overlap(self._h, int(on)), "ovggt_cache_set_overlap")
 
     def profile_enable(self, on: bool) -> None:
         _check(lib().ovggt_cache_profile_enable(self._h, int(on)), "ovggt_cache_profile_enable")

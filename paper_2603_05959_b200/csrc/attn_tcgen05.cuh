@@ -38,7 +38,7 @@ constexpr int kMaxSplits = 16;
 
 struct AttnBarriers {
   unsigned long long q_full, s_full[2], p_full[2], pv_done, o_full, drain;
-  unsigned long long k_full[kKVStages], v_full[kKVStages];
+  unsigned long long k_full[kKVStages], k_empty[kKVStages], v_full[kKVStages], v_empty[kKVStages];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -234,6 +234,8 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     mbar_init(&B->drain, 1);
     for (int s = 0; s < kKVStages; ++s) {
       mbar_init(&B->k_full[s], 1);
+      mbar_init(&B->k_empty[s], 1);
+      mbar_init(&B->v_empty[s], 1);
       mbar_init(&B->v_full[s], 1);
     }
     B->abort_flag = 0;
@@ -264,16 +266,12 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int s = it % kKVStages;
         const uint32_t ph = (uint32_t)(it / kKVStages) & 1u;
         const int row = (t_begin + it) * kBN;
-        // stage s last held the keys of tile it - 2: free once both score MMAs of that tile have completed, which
-        // is what the completion of s_full[1] for that tile says (a commit covers every earlier MMA of the thread)
-        if (it >= kKVStages) ok = mbar_wait(&B->s_full[1], (uint32_t)(it - kKVStages) & 1u, B, P.status);
+        ok = mbar_wait(&B->k_empty[s], ph ^ 1u, B, P.status);
         if (!ok) break;
         mbar_expect_tx(&B->k_full[s], kTileBytes);
         tma_load_2d(sK + s * kTileBytes, &tm_k, h * kHD, row, &B->k_full[s]);
         ++issued_k;
-        // ... and the values of tile it - 2: their last reader, P V of its second half, is issued before the second
-        // score MMA of tile it - 1, so s_full[1] of tile it - 1 covers it
-        if (it >= kKVStages) ok = mbar_wait(&B->s_full[1], (uint32_t)(it - kKVStages + 1) & 1u, B, P.status);
+        ok = mbar_wait(&B->v_empty[s], ph ^ 1u, B, P.status);
         if (!ok) break;
         mbar_expect_tx(&B->v_full[s], kTileBytes);
         tma_load_2d(sV + s * kTileBytes, &tm_v, h * kHD, row, &B->v_full[s]);
@@ -313,6 +311,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         tc_commit(&B->s_full[0]);
         issue_qk(0, 1);
         tc_commit(&B->s_full[1]);
+        tc_commit(&B->k_empty[0]);
       }
       for (int it = 0; it < n_tiles && ok; ++it) {
         const int s = it % kKVStages, s1 = (it + 1) % kKVStages;
@@ -330,6 +329,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           for (int kk = 0; kk < kHalf / 16; ++kk)   // 16 KV rows = 2048 bytes; P: 8 TMEM columns per 16 bf16
             mma_ts(tmem + kColO, tmem + kColS + hf * kHalf + kk * 8, dv + (uint64_t)((hf * (kHalf / 16) + kk) * 128),
                    idesc_pv, (it > 0 || hf > 0 || kk > 0));
+          if (hf == 1) tc_commit(&B->v_empty[s]);
           if (!more && hf == 0) tc_commit(&B->pv_done);   // (the last half has no later score MMA to tell it by)
           if (more) {
             if (hf == 0) {
@@ -339,6 +339,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
             issue_qk(s1, hf);
             tc_commit(&B->s_full[hf]);
+            if (hf == 1) tc_commit(&B->k_empty[s1]);
           }
         }
       }

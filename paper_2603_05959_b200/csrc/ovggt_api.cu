@@ -221,7 +221,8 @@ struct ovggt_cache {
   // ovggt_layer_step scores the cache (diversity, residual norms) on a second, higher-priority stream while the
   // attention runs: the scores do not depend on the attention.  Host objects only; absent if creation failed.
   cudaStream_t side = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_app = nullptr;
+  bool overlap = true;            // ovggt_cache_set_overlap
   // optional per-kernel-class timing (host-side CUDA events; no device memory)
   bool prof = false;
   struct ProfRec { int cls; cudaEvent_t a, b; };
@@ -396,11 +397,13 @@ extern "C" int ovggt_cache_create(const ovggt_config* cfg, ovggt_cache** out) {
     if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess ||
         cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, hi) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_app, cudaEventDisableTiming) != cudaSuccess) {
       if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+      if (h->ev_join) cudaEventDestroy(h->ev_join);
       if (h->side) cudaStreamDestroy(h->side);
       h->side = nullptr;
-      h->ev_fork = h->ev_join = nullptr;
+      h->ev_fork = h->ev_join = h->ev_app = nullptr;
       (void)cudaGetLastError();
     }
   }
@@ -425,12 +428,15 @@ extern "C" int ovggt_cache_destroy(ovggt_cache* h) {
     cudaStreamDestroy(h->side);
     cudaEventDestroy(h->ev_fork);
     cudaEventDestroy(h->ev_join);
+    cudaEventDestroy(h->ev_app);
   }
   delete h;
   return OVGGT_OK;
 }
 
-extern "C" int ovggt_layer_attend(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
+namespace {
+// Eq. 2: validation of the attend half and the append itself.
+int enqueue_append(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st) {
   int rc = check_layer(h, layer);
   if (rc) return rc;
   if (!io || !io->q || !io->k || !io->v || !io->out) return OVGGT_ERR_INVALID_ARG;
@@ -439,19 +445,24 @@ extern "C" int ovggt_layer_attend(ovggt_cache* h, int32_t layer, const ovggt_fra
   if (S.pending) return OVGGT_ERR_FRAME_ORDER;
   if (S.frames_seen > 0 && io->frame_id <= S.pending_frame) return OVGGT_ERR_FRAME_ORDER;
   if (io->frame_id < 0 || (h->first_frame >= 0 && io->frame_id < h->first_frame)) return OVGGT_ERR_FRAME_ORDER;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   h->last_stream = st;
   const int M = h->M, C = h->C, nvec = C * h->elem / 16, b = S.cur;
   const int grid = std::min((2 * M + 7) / 8, 148 * 8);
-  {
-    ProfScope ps(h, OVGGT_PROF_APPEND, st);
-    k_append<<<grid, 256, 0, st>>>((const uint4*)io->k, (const uint4*)io->v, M, nvec, S.n, (long long)io->frame_id,
-                                   (uint4*)S.kbuf[b], (uint4*)S.vbuf[b], S.ids[b], S.flags[b], S.stored[b]);
-    LAUNCHED();
-  }
+  ProfScope ps(h, OVGGT_PROF_APPEND, st);
+  k_append<<<grid, 256, 0, st>>>((const uint4*)io->k, (const uint4*)io->v, M, nvec, S.n, (long long)io->frame_id,
+                                 (uint4*)S.kbuf[b], (uint4*)S.vbuf[b], S.ids[b], S.flags[b], S.stored[b]);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
+// The attention over all n + M rows, and the bookkeeping that closes the attend half.
+int enqueue_attention(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st) {
+  LayerState& S = h->layers[layer];
+  const int b = S.cur;
+  int rc;
   {
     ProfScope ps(h, OVGGT_PROF_ATTENTION, st);
-    rc = launch_attention(io->q, S.kbuf[b], S.vbuf[b], M, S.n + M, h->cfg.n_heads, h->cfg.dtype, io->out,
+    rc = launch_attention(io->q, S.kbuf[b], S.vbuf[b], h->M, S.n + h->M, h->cfg.n_heads, h->cfg.dtype, io->out,
                           h->attn_scratch, h->status, st);
   }
   if (rc) return rc;
@@ -462,6 +473,14 @@ extern "C" int ovggt_layer_attend(ovggt_cache* h, int32_t layer, const ovggt_fra
   S.pending = true;
   S.pending_frame = io->frame_id;
   return OVGGT_OK;
+}
+}  // namespace
+
+extern "C" int ovggt_layer_attend(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = enqueue_append(h, layer, io, st);
+  if (rc) return rc;
+  return enqueue_attention(h, layer, io, st);
 }
 
 extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
@@ -500,7 +519,7 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
   const bool prelaunched = S.scores_frame == t;    // ovggt_layer_step already enqueued them on the side stream
   S.scores_frame = -1;
   if (prelaunched) {
-    CK(cudaStreamWaitEvent(st, h->ev_join, 0));
+    // (enqueued earlier on this same stream by ovggt_layer_step)
   } else if (!fused_scores) {
     ProfScope ps(h, OVGGT_PROF_ROW_NORMS, st);
     rc = launch_row_norms(io->resid, M, C, c.dtype, S.s_raw, st);
@@ -570,39 +589,52 @@ extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame
   int rc = check_layer(h, layer);
   if (rc) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // The scores of the cached rows (key diversity) and of the new rows (residual norms) depend on neither the
-  // append nor the attention of this step: start them now on the side stream, join before the selection.
-  bool pre = false;
-  if (h->side && io && io->resid && aligned16(io->resid) && io->q && io->k && io->v && io->out) {
-    LayerState& S = h->layers[layer];
-    const ovggt_config& c = h->cfg;
-    if (!S.pending && c.score_mode == OVGGT_SCORE_HYBRID && S.n > 0 && S.colsum_nparts > 0 &&
-        io->frame_id > S.pending_frame) {
-      CK(cudaEventRecord(h->ev_fork, st));
-      CK(cudaStreamWaitEvent(h->side, h->ev_fork, 0));
-      {
-        ProfScope ps(h, OVGGT_PROF_DIVERSITY, h->side);
-        rc = launch_diversity_from_parts(S.kbuf[S.cur], S.n, h->C, c.dtype, S.colsum_part, S.colsum_nparts, h->ksum,
-                                         S.d, io->resid, h->M, S.s_raw, h->side);
-      }
-      CK(cudaEventRecord(h->ev_join, h->side));
-      if (rc) {
-        (void)cudaStreamWaitEvent(st, h->ev_join, 0);
-        return rc;
-      }
-      S.scores_frame = io->frame_id;
-      pre = true;
-    }
+  const bool can_overlap = h->side && h->overlap && io && io->resid && aligned16(io->resid) && io->q && io->k &&
+                           io->v && io->out && !h->layers[layer].pending;
+  if (!can_overlap) {
+    rc = ovggt_layer_attend(h, layer, io, stream);
+    if (rc) return rc;
+    return ovggt_layer_compress(h, layer, io, stream);
   }
-  rc = ovggt_layer_attend(h, layer, io, stream);
-  if (rc) {
-    if (pre) {                          // keep the caller's stream ordered after the side work
-      (void)cudaStreamWaitEvent(st, h->ev_join, 0);
-      h->layers[layer].scores_frame = -1;
+  // Scoring, selection and compaction (Eq. 5-8) read the cache and the new rows but not the attention's output, and
+  // the attention only reads the buffers the compaction reads.  So the compress half runs on the handle's second,
+  // higher-priority stream beside the attention:
+  //   stream:  fork ........ append . fork' ........ attention ................................ join
+  //   side:         scores (diversity, norms) ....... [after fork'] selection, compaction ......./
+  LayerState& S = h->layers[layer];
+  const ovggt_config& c = h->cfg;
+  CK(cudaEventRecord(h->ev_fork, st));
+  CK(cudaStreamWaitEvent(h->side, h->ev_fork, 0));
+  if (c.score_mode == OVGGT_SCORE_HYBRID && S.n > 0 && S.colsum_nparts > 0 && io->frame_id > S.pending_frame) {
+    {
+      ProfScope ps(h, OVGGT_PROF_DIVERSITY, h->side);
+      rc = launch_diversity_from_parts(S.kbuf[S.cur], S.n, h->C, c.dtype, S.colsum_part, S.colsum_nparts, h->ksum,
+                                       S.d, io->resid, h->M, S.s_raw, h->side);
     }
-    return rc;
+    if (rc == OVGGT_OK) S.scores_frame = io->frame_id;
   }
-  return ovggt_layer_compress(h, layer, io, stream);
+  if (rc == OVGGT_OK) rc = enqueue_append(h, layer, io, st);
+  if (rc == OVGGT_OK) {
+    CK(cudaEventRecord(h->ev_app, st));
+    CK(cudaStreamWaitEvent(h->side, h->ev_app, 0));
+    rc = enqueue_attention(h, layer, io, st);
+  }
+  if (rc == OVGGT_OK) rc = ovggt_layer_compress(h, layer, io, h->side);
+  // join: whatever happened, the caller's stream is ordered after the side work
+  S.scores_frame = -1;
+  h->last_stream = st;
+  cudaError_t e1 = cudaEventRecord(h->ev_join, h->side);
+  cudaError_t e2 = cudaStreamWaitEvent(st, h->ev_join, 0);
+  if (rc) return rc;
+  if (e1 != cudaSuccess) return cuda_fail(e1);
+  if (e2 != cudaSuccess) return cuda_fail(e2);
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_cache_set_overlap(ovggt_cache* h, int32_t enable) {
+  if (!h) return OVGGT_ERR_INVALID_ARG;
+  h->overlap = enable != 0;
+  return OVGGT_OK;
 }
 
 extern "C" int ovggt_layer_step_host(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {

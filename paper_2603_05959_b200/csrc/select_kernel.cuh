@@ -17,7 +17,7 @@ namespace ovggt {
 
 namespace cg = cooperative_groups;
 
-constexpr int kSelectThreads = 1024;
+constexpr int kSelectThreads = 512;   // 512 x 64 registers: half an SM, so a CTA fits beside an attention CTA
 constexpr int kSelectMaxCtas = 8;
 constexpr uint32_t kKeyProtected = 0xFFFFFFFFu;   // above the key of +inf (0xFF800000)
 
