@@ -136,10 +136,13 @@ int ovggt_layer_step(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io
  * other on `stream`, which is what per-kernel timing wants. */
 int ovggt_cache_set_overlap(ovggt_cache* cache, int32_t enable);
 
-/* The same step with HOST tensors: q, k, v, resid, conf, out are host pointers (pinned memory
- * makes the copies asynchronous); score_override must be NULL.  The inputs are copied into staging
- * buffers of the workspace, the step runs, and out is copied back, all on `stream`.  The call returns
- * without synchronising: out is valid once the stream has been synchronised. */
+/* The same step with HOST tensors: q, k, v, resid, conf, out are host pointers; score_override must be NULL.
+ * The host inputs must hold their values when the call is made.  They are copied into one of two sets of staging
+ * buffers of the workspace on a copy stream the handle owns (not ordered after earlier work on `stream`), so with
+ * pinned host memory the copies of one step overlap the kernels of the step before; the step itself runs on
+ * `stream`; out is written by the kernel itself when it is pinned, mapped host memory, and copied back on `stream`
+ * otherwise.  The call returns without synchronising: once `stream` has been synchronised, out is valid and the
+ * input buffers may be reused. */
 int ovggt_layer_step_host(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
 
 /* Counters of one layer.  Synchronises the stream the handle last used (to read the device status word). */

@@ -213,8 +213,13 @@ struct ovggt_cache {
   float *colsum_part = nullptr, *ksum = nullptr;
   void* attn_scratch = nullptr;
   int* status = nullptr;
-  char *stage_q = nullptr, *stage_k = nullptr, *stage_v = nullptr, *stage_r = nullptr, *stage_o = nullptr;
-  float* stage_conf = nullptr;
+  // two sets of staging buffers for ovggt_layer_step_host: the copies of one step overlap the kernels of the step before
+  char *stage_q[2] = {}, *stage_k[2] = {}, *stage_v[2] = {}, *stage_r[2] = {}, *stage_o[2] = {};
+  float* stage_conf[2] = {};
+  int stage_next = 0;
+  cudaStream_t copy = nullptr;                       // host -> device copies of ovggt_layer_step_host
+  cudaEvent_t ev_h2d[2] = {}, ev_done[2] = {};       // set p: inputs have arrived / the step that read them is done
+  bool stage_used[2] = {false, false};
   float w_center = 0, w_edge = 0, w_corner = 0;
   cudaStream_t last_stream = nullptr;
   int max_rows = 0;
@@ -333,20 +338,24 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
   const size_t o_ksum = L.take((size_t)kColsumSlices * C * 4);
   const size_t o_attn = L.take(ovggt_k_attention_scratch_bytes(M, max_rows, c->n_heads));
   const size_t o_status = L.take(64);
-  size_t o_stage[5];
-  for (int i = 0; i < 5; ++i) o_stage[i] = L.take((size_t)M * C * eb);
-  const size_t o_conf = L.take((size_t)Np * 4);
+  size_t o_stage[2][5], o_conf[2];
+  for (int p = 0; p < 2; ++p) {
+    for (int i = 0; i < 5; ++i) o_stage[p][i] = L.take((size_t)M * C * eb);
+    o_conf[p] = L.take((size_t)Np * 4);
+  }
   if (h) {
     h->colsum_part = reinterpret_cast<float*>(base + o_part);
     h->ksum = reinterpret_cast<float*>(base + o_ksum);
     h->attn_scratch = base + o_attn;
     h->status = reinterpret_cast<int*>(base + o_status);
-    h->stage_q = base + o_stage[0];
-    h->stage_k = base + o_stage[1];
-    h->stage_v = base + o_stage[2];
-    h->stage_r = base + o_stage[3];
-    h->stage_o = base + o_stage[4];
-    h->stage_conf = reinterpret_cast<float*>(base + o_conf);
+    for (int p = 0; p < 2; ++p) {
+      h->stage_q[p] = base + o_stage[p][0];
+      h->stage_k[p] = base + o_stage[p][1];
+      h->stage_v[p] = base + o_stage[p][2];
+      h->stage_r[p] = base + o_stage[p][3];
+      h->stage_o[p] = base + o_stage[p][4];
+      h->stage_conf[p] = reinterpret_cast<float*>(base + o_conf[p]);
+    }
     h->max_rows = max_rows;
   }
   return align_up(L.total, 1024);
@@ -407,6 +416,22 @@ extern "C" int ovggt_cache_create(const ovggt_config* cfg, ovggt_cache** out) {
       (void)cudaGetLastError();
     }
   }
+  {
+    bool ok = cudaStreamCreateWithFlags(&h->copy, cudaStreamNonBlocking) == cudaSuccess;
+    for (int p = 0; p < 2 && ok; ++p)
+      ok = cudaEventCreateWithFlags(&h->ev_h2d[p], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&h->ev_done[p], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      for (int p = 0; p < 2; ++p) {
+        if (h->ev_h2d[p]) cudaEventDestroy(h->ev_h2d[p]);
+        if (h->ev_done[p]) cudaEventDestroy(h->ev_done[p]);
+        h->ev_h2d[p] = h->ev_done[p] = nullptr;
+      }
+      if (h->copy) cudaStreamDestroy(h->copy);
+      h->copy = nullptr;
+      (void)cudaGetLastError();
+    }
+  }
   cudaError_t e = cudaMemset(h->status, 0, 64);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
@@ -422,6 +447,14 @@ extern "C" int ovggt_cache_destroy(ovggt_cache* h) {
   for (auto& r : h->prof_recs) {
     cudaEventDestroy(r.a);
     cudaEventDestroy(r.b);
+  }
+  if (h->copy) {
+    cudaStreamSynchronize(h->copy);
+    cudaStreamDestroy(h->copy);
+    for (int p = 0; p < 2; ++p) {
+      cudaEventDestroy(h->ev_h2d[p]);
+      cudaEventDestroy(h->ev_done[p]);
+    }
   }
   if (h->side) {
     cudaStreamSynchronize(h->side);
@@ -643,19 +676,50 @@ extern "C" int ovggt_layer_step_host(ovggt_cache* h, int32_t layer, const ovggt_
   if (!io || !io->q || !io->k || !io->v || !io->resid || !io->out || io->score_override) return OVGGT_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t bytes = (size_t)h->M * h->C * h->elem;
-  CK(cudaMemcpyAsync(h->stage_q, io->q, bytes, cudaMemcpyHostToDevice, st));
-  CK(cudaMemcpyAsync(h->stage_k, io->k, bytes, cudaMemcpyHostToDevice, st));
-  CK(cudaMemcpyAsync(h->stage_v, io->v, bytes, cudaMemcpyHostToDevice, st));
-  CK(cudaMemcpyAsync(h->stage_r, io->resid, bytes, cudaMemcpyHostToDevice, st));
-  if (io->conf) CK(cudaMemcpyAsync(h->stage_conf, io->conf, (size_t)h->Np * 4, cudaMemcpyHostToDevice, st));
+  // Inputs go through one of two staging sets on a copy stream of the handle's own, so that the copies of this
+  // step run while the kernels of the previous step (enqueued on `stream` by the previous call) still compute.
+  const int p = h->stage_next;
+  h->stage_next ^= 1;
+  cudaStream_t cs = h->copy ? h->copy : st;
+  if (h->copy) {
+    // the set was last read by the step two calls ago
+    if (h->stage_used[p]) CK(cudaStreamWaitEvent(cs, h->ev_done[p], 0));
+  }
+  CK(cudaMemcpyAsync(h->stage_q[p], io->q, bytes, cudaMemcpyHostToDevice, cs));
+  CK(cudaMemcpyAsync(h->stage_k[p], io->k, bytes, cudaMemcpyHostToDevice, cs));
+  CK(cudaMemcpyAsync(h->stage_v[p], io->v, bytes, cudaMemcpyHostToDevice, cs));
+  CK(cudaMemcpyAsync(h->stage_r[p], io->resid, bytes, cudaMemcpyHostToDevice, cs));
+  if (io->conf) CK(cudaMemcpyAsync(h->stage_conf[p], io->conf, (size_t)h->Np * 4, cudaMemcpyHostToDevice, cs));
+  if (h->copy) {
+    CK(cudaEventRecord(h->ev_h2d[p], cs));
+    CK(cudaStreamWaitEvent(st, h->ev_h2d[p], 0));
+  }
   ovggt_frame_io dev = *io;
-  dev.q = h->stage_q; dev.k = h->stage_k; dev.v = h->stage_v; dev.resid = h->stage_r;
-  dev.conf = io->conf ? h->stage_conf : nullptr;
-  dev.out = h->stage_o;
+  dev.q = h->stage_q[p]; dev.k = h->stage_k[p]; dev.v = h->stage_v[p]; dev.resid = h->stage_r[p];
+  dev.conf = io->conf ? h->stage_conf[p] : nullptr;
+  // Pinned, mapped host memory can take the output straight from the kernel (posted writes over the bus, no
+  // separate copy after the step); anything else goes through the staging buffer.
+  void* out_dev = nullptr;
+  {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, io->out) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+        attr.devicePointer != nullptr && aligned16(attr.devicePointer))
+      out_dev = attr.devicePointer;
+    else
+      (void)cudaGetLastError();
+  }
+  dev.out = out_dev ? out_dev : h->stage_o[p];
   rc = ovggt_layer_step(h, layer, &dev, stream);
-  if (rc) return rc;
-  CK(cudaMemcpyAsync(io->out, h->stage_o, bytes, cudaMemcpyDeviceToHost, st));
-  return OVGGT_OK;
+  if (rc == OVGGT_OK && !out_dev) {
+    cudaError_t e = cudaMemcpyAsync(io->out, h->stage_o[p], bytes, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) rc = cuda_fail(e);
+  }
+  if (h->copy) {
+    cudaError_t e = cudaEventRecord(h->ev_done[p], st);
+    if (e != cudaSuccess && rc == OVGGT_OK) rc = cuda_fail(e);
+    h->stage_used[p] = true;
+  }
+  return rc;
 }
 
 extern "C" int ovggt_cache_stats(ovggt_cache* h, int32_t layer, ovggt_stats* out) {

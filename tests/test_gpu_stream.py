@@ -163,18 +163,29 @@ def test_call_order_errors():
     c.destroy()
 
 
-def test_host_buffer_entry_point_matches_device_entry_point():
+@pytest.mark.parametrize("pin", [True, False])
+def test_host_buffer_entry_point_matches_device_entry_point(pin):
+    """Pinned buffers: staged copies on the handle's copy stream, output written by the kernel into host memory.
+    Pageable buffers: the output comes back through the staging buffer.  Several calls are in flight before the
+    first synchronisation, so both staging sets are in use."""
     cfg = gen.StreamConfig(name="mid", n_heads=2, grid_h=9, grid_w=10, budget=300, anchor_tokens=4,
-                           min_anchor_interval=2, tau=0.5, n_frames=6)
+                           min_anchor_interval=2, tau=0.5, n_frames=7)
     a, b = B.OvggtCache.from_stream(cfg), B.OvggtCache.from_stream(cfg)
+    host = [DeviceFrame(cfg, gen.frame_inputs(cfg, t), None, pin=pin) for t in range(cfg.n_frames)]
+    outs_b = []
+    for t in range(cfg.n_frames):                        # no synchronisation between the calls
+        h = host[t]
+        ob = torch.empty((cfg.tokens_per_frame, cfg.dim), dtype=torch.bfloat16)
+        ob = ob.pin_memory() if pin else ob
+        b.layer_step_host(0, t, h.q, h.k, h.v, h.resid, h.conf, h.rho, ob)
+        outs_b.append(ob)
+    torch.cuda.synchronize()
     for t in range(cfg.n_frames):
         fi = gen.frame_inputs(cfg, t)
-        d, h = DeviceFrame(cfg, fi, "cuda"), DeviceFrame(cfg, fi, None, pin=True)
+        d = DeviceFrame(cfg, fi, "cuda")
         oa = a.layer_step(0, t, d.q, d.k, d.v, d.resid, d.conf, d.rho)
-        ob = torch.empty((cfg.tokens_per_frame, cfg.dim), dtype=oa.dtype).pin_memory()
-        b.layer_step_host(0, t, h.q, h.k, h.v, h.resid, h.conf, h.rho, ob)
         torch.cuda.synchronize()
-        assert torch.equal(oa.cpu(), ob)
+        assert torch.equal(oa.cpu(), outs_b[t]), t
     ea, eb = a.export(0), b.export(0)
     for key in ea:
         assert np.array_equal(ea[key], eb[key])
