@@ -223,7 +223,12 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const int n_tiles = min(P.tiles_total, t_begin + P.tiles_per_split) - t_begin;   // >= 1 by construction
   const int C = P.H * kHD;
 
-  if (threadIdx.x == 0) {
+  // The producer's elected thread sets the barriers up and sends the first loads (Q and the first K/V tile) on their
+  // way at once, so that they travel while tensor memory is allocated and the CTA meets at its first barrier.
+  if (warp == 4 && lane == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_q) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_k) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_v) : "memory");
     mbar_init(&B->q_full, 1);
     for (int hf = 0; hf < 2; ++hf) {
       mbar_init(&B->s_full[hf], 1);
@@ -241,6 +246,12 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     B->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    mbar_expect_tx(&B->q_full, kTileBytes);
+    tma_load_2d(sQ, &tm_q, h * kHD, qt * kBM, &B->q_full);
+    mbar_expect_tx(&B->k_full[0], kTileBytes);
+    tma_load_2d(sK, &tm_k, h * kHD, t_begin * kBN, &B->k_full[0]);
+    mbar_expect_tx(&B->v_full[0], kTileBytes);
+    tma_load_2d(sV, &tm_v, h * kHD, t_begin * kBN, &B->v_full[0]);
   }
   if (warp == 5) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&B->tmem_base)),
@@ -258,11 +269,9 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   if (warp == 4) {
     // ------------------------------------------------ TMA producer
     if (lane == 0) {
-      int issued_k = 0, issued_v = 0;
+      int issued_k = 1, issued_v = 1;                // Q and tile 0 were sent during set-up
       bool ok = true;
-      mbar_expect_tx(&B->q_full, kTileBytes);
-      tma_load_2d(sQ, &tm_q, h * kHD, qt * kBM, &B->q_full);
-      for (int it = 0; it < n_tiles && ok; ++it) {
+      for (int it = 1; it < n_tiles && ok; ++it) {
         const int s = it % kKVStages;
         const uint32_t ph = (uint32_t)(it / kKVStages) & 1u;
         const int row = (t_begin + it) * kBN;
