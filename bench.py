@@ -245,6 +245,7 @@ def run_ours(args) -> None:
     import torch
     import torch.distributed as dist
     from paper_2603_05959_b200 import binding as B
+    from paper_2603_05959_b200 import replicas
     from paper_2603_05959_b200.stream import DeviceFrame
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -257,7 +258,7 @@ def run_ours(args) -> None:
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    cfg = workload_config(seed_offset=rank)
+    cfg = workload_config(seed_offset=replicas.rank_seed(0, rank))
     M, C, Bud = cfg.tokens_per_frame, cfg.dim, cfg.budget
     K, W = args.steps, args.warmup
     fill = -(-Bud // M) + 1                           # frames until the cache is full, plus one
@@ -332,12 +333,9 @@ def run_ours(args) -> None:
     assert st["device_status"] == 0 and st["n_cached"] == Bud
 
     # ---- max over ranks
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
-    value = world * K / (total_ms * 1e-3)
-    e2e_value = world * n_e2e / (e2e_ms * 1e-3)
+    total_ms, e2e_ms = replicas.max_over_ranks([total_ms, e2e_ms], world, dev)
+    value = replicas.aggregate_rate(K, total_ms, world)
+    e2e_value = replicas.aggregate_rate(n_e2e, e2e_ms, world)
 
     if rank == 0:
         peaks, peak_kind = load_peaks()
