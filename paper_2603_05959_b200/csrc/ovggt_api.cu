@@ -108,22 +108,26 @@ int launch_diversity(const void* K, int rows, int C, int dtype, float* part, flo
 constexpr int kColsumSlices = 8;
 
 // Diversity from the per-CTA column sums the last compaction left (nparts rows of part): no pass over K for the sums.
-// slices: [kColsumSlices, C] floats.
+// slices: [kColsumSlices, C] floats of scratch, then the column sums [C], then one arrival counter per 32 columns
+// (colsum_scratch_bytes(C) in all; the counters zero before the first use).
+size_t colsum_scratch_bytes(int C) { return ((size_t)(kColsumSlices + 1) * C * 4 + ((size_t)(C + 31) / 32) * 4 + 255) / 256 * 256; }
 // The same launch also computes the residual norms s_raw [resid_rows] of the new frame when resid is given.
 int launch_diversity_from_parts(const void* K, int rows, int C, int dtype, const float* part, int nparts, float* slices,
                                 float* d, const void* resid, int resid_rows, float* s_raw, cudaStream_t st) {
   if (rows <= 0) return OVGGT_OK;
   const int nvec = C * elem_bytes(dtype) / 16;
-  k_colsum_final_sliced<<<dim3((C + 31) / 32, kColsumSlices), 1024, 0, st>>>(part, nparts, C, slices);
+  float* ksum = slices + (size_t)kColsumSlices * C;
+  int* arrived = reinterpret_cast<int*>(ksum + C);
+  k_colsum_final_sliced<<<dim3((C + 31) / 32, kColsumSlices), 1024, 0, st>>>(part, nparts, C, slices, ksum, arrived);
   LAUNCHED();
   const int grid = std::min((rows + 15) / 16, 148 * 8);
   const size_t smem = (size_t)C * 4;
   const int norm_ctas = resid ? (resid_rows + 7) / 8 : 0;
   if (dtype == kBF16)
-    k_diversity<kBF16><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, slices, kColsumSlices, d, grid,
+    k_diversity<kBF16><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d, grid,
                                                             (const uint4*)resid, resid_rows, s_raw);
   else
-    k_diversity<kF32><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, slices, kColsumSlices, d, grid,
+    k_diversity<kF32><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d, grid,
                                                            (const uint4*)resid, resid_rows, s_raw);
   LAUNCHED();
   return OVGGT_OK;
@@ -335,7 +339,7 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
     }
   }
   const size_t o_part = L.take((size_t)kMaxColsumParts * C * 4);
-  const size_t o_ksum = L.take((size_t)kColsumSlices * C * 4);
+  const size_t o_ksum = L.take(colsum_scratch_bytes(C));
   const size_t o_attn = L.take(ovggt_k_attention_scratch_bytes(M, max_rows, c->n_heads));
   const size_t o_status = L.take(64);
   size_t o_stage[2][5], o_conf[2];
@@ -433,6 +437,7 @@ extern "C" int ovggt_cache_create(const ovggt_config* cfg, ovggt_cache** out) {
     }
   }
   cudaError_t e = cudaMemset(h->status, 0, 64);
+  if (e == cudaSuccess) e = cudaMemset(h->ksum, 0, colsum_scratch_bytes(h->C));   // (its arrival counters)
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     delete h;

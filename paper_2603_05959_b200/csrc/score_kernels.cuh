@@ -98,11 +98,13 @@ __global__ void __launch_bounds__(1024) k_colsum_final(const float* __restrict__
 }
 
 // Stage 2 for many partials (the compaction kernel leaves one per CTA): CTA (x, y) folds the partials
-// p = y, y + gridDim.y, ... of its 32 columns the same way; ksum8[y, c] holds the result and the diversity kernel
-// folds the gridDim.y slices in order when it stages the sums.
+// p = y, y + gridDim.y, ... of its 32 columns into slice y; the CTA of a column block that finishes last folds the
+// gridDim.y slices, in slice order, into ksum.  arrived: one counter per column block, zero before and after.
 __global__ void __launch_bounds__(1024) k_colsum_final_sliced(const float* __restrict__ part, int nparts, int C,
-                                                              float* __restrict__ ksum_slices) {
+                                                              float* __restrict__ ksum_slices,
+                                                              float* __restrict__ ksum, int* __restrict__ arrived) {
   __shared__ float sh[32][33];
+  __shared__ int is_last;
   const int cx = threadIdx.x & 31, py = threadIdx.x >> 5;
   const int c = blockIdx.x * 32 + cx;
   float acc = 0.0f;
@@ -117,6 +119,20 @@ __global__ void __launch_bounds__(1024) k_colsum_final_sliced(const float* __res
 #pragma unroll
     for (int i = 0; i < 32; ++i) t += sh[i][cx];
     ksum_slices[(size_t)blockIdx.y * C + c] = t;
+    __threadfence();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int old = atomicAdd(&arrived[blockIdx.x], 1);
+    is_last = old == (int)gridDim.y - 1;
+    if (is_last) arrived[blockIdx.x] = 0;
+  }
+  __syncthreads();
+  if (is_last && py == 0 && c < C) {
+    __threadfence();
+    float t = 0.0f;
+    for (int y = 0; y < (int)gridDim.y; ++y) t += __ldcg(&ksum_slices[(size_t)y * C + c]);
+    ksum[c] = t;
   }
 }
 
