@@ -216,3 +216,36 @@ def test_config2_full_size_stream_teacher_forced():
     rows = np.sort(np.random.default_rng(11).choice(cfg.tokens_per_frame, 16, replace=False)).astype(np.int32)
     threads = max(1, min(32, torch.get_num_threads()))
     run_teacher_forced(cfg, 40, attn_frames={0, 11, 12, 39}, attn_rows=rows, export_every=13, threads=threads)
+
+
+def test_config2_full_size_through_layer_step_with_overlap():
+    """The call the benchmark times: ovggt_layer_step on the benchmark configuration, where the compress half runs
+    beside the attention on the handle's second stream.  Teacher-forced, so survivors and layout are bit-exact;
+    the attention is checked on sampled rows while the compress half is running next to it."""
+    cfg = gen.config_vggt_layer()
+    orc.set_threads(max(1, min(32, torch.get_num_threads())))
+    rows = np.sort(np.random.default_rng(12).choice(cfg.tokens_per_frame, 12, replace=False)).astype(np.int32)
+    layer = orc.OracleLayer.from_stream(cfg)
+    cache = B.OvggtCache.from_stream(cfg)
+    for t in range(16):
+        fi = gen.frame_inputs(cfg, t)
+        df = DeviceFrame(cfg, fi, "cuda")
+        check = t in (0, 12, 15)
+        ref_out = layer.attend(t, fi.q, fi.k, fi.v, rows=rows, compute=check)
+        ref = layer.compress(fi.resid, fi.conf, fi.rho)
+        out = cache.layer_step(0, t, df.q, df.k, df.v, df.resid, df.conf, df.rho,
+                               score_override=torch.from_numpy(ref["r"]).cuda())
+        sel = cache.last_selection(0)
+        np.testing.assert_array_equal(sel["survivors"], ref["survivors"], err_msg=f"frame {t}")
+        fin = np.isfinite(ref["r"])
+        np.testing.assert_allclose(sel["r"][fin], ref["r"][fin], rtol=0, atol=R_ATOL, err_msg=f"frame {t}")
+        if check:
+            err = np.abs(out_to_f32(out)[rows] - ref_out)
+            assert err.max() <= ATT_MAX and err.mean() <= ATT_MEAN, (t, err.max(), err.mean())
+    ex, rx = cache.export(0), layer.export()
+    np.testing.assert_array_equal(ex["ids"], rx["ids"])
+    np.testing.assert_array_equal(ex["flags"], rx["flags"])
+    assert np.array_equal(storage_to_f32(ex["k"], cfg.dtype), rx["k"])
+    assert np.array_equal(storage_to_f32(ex["v"], cfg.dtype), rx["v"])
+    assert cache.stats(0)["device_status"] == 0
+    cache.destroy()
