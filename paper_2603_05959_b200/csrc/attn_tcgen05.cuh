@@ -24,15 +24,17 @@
 namespace ovggt {
 
 constexpr int kBM = 128;            // query rows per CTA
-constexpr int kBN = 128;            // KV rows per tile
+constexpr int kBN = 192;            // KV rows per tile
+constexpr int kCtasPerSm = 2;       // resident CTAs per SM
 constexpr int kHD = 64;             // head dim
 constexpr int kKVStages = 2;
 constexpr int kAttnThreads = 256;
 constexpr int kRegsSoftmax = 216, kRegsOther = 40;   // 2 CTAs x (128 x 216 + 128 x 40) = 64K registers
-constexpr int kTileBytes = kBN * kHD * 2;          // 16 KB
+constexpr int kQBytes = kBM * kHD * 2;           // 16 KB
+constexpr int kTileBytes = kBN * kHD * 2;          // 24 KB
 constexpr int kHalf = kBN / 2;      // KV rows per S buffer
 constexpr int kTmemCols = 256;
-constexpr int kColS = 0, kColO = 128;   // S_0 at columns [0, 64), S_1 at [64, 128), O at [128, 192)
+constexpr int kColS = 0, kColO = 2 * kHalf;   // S_0 at columns [0, 96), S_1 at [96, 192), O at [192, 256): all 256 columns
 constexpr float kRescaleThreshold = 8.0f;          // log2 units
 constexpr int kMaxSplits = 16;
 
@@ -43,7 +45,8 @@ struct AttnBarriers {
   int abort_flag;
 };
 
-constexpr size_t kAttnSmemBytes = 1024 + (size_t)kTileBytes * (1 + 2 * kKVStages) + sizeof(AttnBarriers) + 64;
+// (no slack for aligning the base by hand: two CTAs of 114.9 KB must fit one SM; the base is checked instead)
+constexpr size_t kAttnSmemBytes = (size_t)kQBytes + (size_t)kTileBytes * 2 * kKVStages + sizeof(AttnBarriers) + 64;
 
 // ---------------------------------------------------------------- PTX wrappers
 
@@ -160,6 +163,23 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
       "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -190,6 +210,14 @@ __device__ __forceinline__ float2 add2(float2 a, float2 b) {
       : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
   return d;
 }
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t d;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
@@ -207,13 +235,16 @@ struct AttnParams {
   int* status;
 };
 
-__global__ void __launch_bounds__(kAttnThreads, 2)
+__global__ void __launch_bounds__(kAttnThreads, kCtasPerSm)
 k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const AttnParams P) {
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  extern __shared__ __align__(1024) unsigned char smem[];
+  if (smem_u32(smem) & 1023u) {                      // the 128-byte swizzle needs 1024-byte aligned tiles
+    if (threadIdx.x == 0) atomicCAS(P.status, 0, OVGGT_ERR_DEVICE_STATUS);
+    return;
+  }
   unsigned char* sQ = smem;
-  unsigned char* sK = sQ + kTileBytes;
+  unsigned char* sK = sQ + kQBytes;
   unsigned char* sV = sK + kKVStages * kTileBytes;
   AttnBarriers* B = reinterpret_cast<AttnBarriers*>(sV + kKVStages * kTileBytes);
 
@@ -246,7 +277,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     B->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    mbar_expect_tx(&B->q_full, kTileBytes);
+    mbar_expect_tx(&B->q_full, kQBytes);
     tma_load_2d(sQ, &tm_q, h * kHD, qt * kBM, &B->q_full);
     mbar_expect_tx(&B->k_full[0], kTileBytes);
     tma_load_2d(sK, &tm_k, h * kHD, t_begin * kBN, &B->k_full[0]);
@@ -301,63 +332,78 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // Issue order (the tensor pipe executes one thread's MMAs in order):
     //   QK(0,0) QK(0,1) | PV(0,0) QK(1,0) PV(0,1) QK(1,1) | PV(1,0) QK(2,0) PV(1,1) QK(2,1) | ...
     // QK(t+1,h) overwrites S_h only after PV(t,h) has read P_h from it.
-    if (lane == 0) {
+    // The whole warp walks the loop in step (every wait result goes through a vote, the tensor-memory base through
+    // a warp reduction), so addresses and descriptors are warp-uniform values; one elected lane issues.
+    {
+      const bool leader = elect_one();
+      const uint32_t tm = __reduce_or_sync(0xFFFFFFFFu, tmem);
       constexpr uint32_t idesc_qk = idesc_bf16(kHalf, false);
       constexpr uint32_t idesc_pv = idesc_bf16(kHD, true);
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ));
-      // S_hf = Q K_hf^T for the KV tile held in stage `st` (64 rows = 8 swizzle groups = 8192 bytes per half)
+      // S_hf = Q K_hf^T for the KV tile held in stage `st` (8 rows = one 1024-byte swizzle group)
       auto issue_qk = [&](int st, int hf) {
         const uint64_t dk = smem_desc_sw128(smem_u32(sK + st * kTileBytes + hf * (kTileBytes / 2)));
+        if (leader) {
 #pragma unroll
-        for (int kk = 0; kk < kHD / 16; ++kk)     // 16 elements of head dim = 32 bytes inside the swizzled row
-          mma_ss(tmem + kColS + hf * kHalf, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_qk, kk > 0);
+          for (int kk = 0; kk < kHD / 16; ++kk)     // 16 elements of head dim = 32 bytes inside the swizzled row
+            mma_ss(tm + kColS + hf * kHalf, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_qk, kk > 0);
+        }
       };
-      bool ok = mbar_wait(&B->q_full, 0, B, P.status);
-      if (ok) ok = mbar_wait(&B->k_full[0], 0, B, P.status);
+      auto wait_all = [&](void* bar, uint32_t parity) {
+        return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, B, P.status)) != 0;
+      };
+      bool ok = wait_all(&B->q_full, 0);
+      if (ok) ok = wait_all(&B->k_full[0], 0);
       if (ok) {
         tc_fence_after();
         issue_qk(0, 0);
-        tc_commit(&B->s_full[0]);
+        if (leader) tc_commit(&B->s_full[0]);
         issue_qk(0, 1);
-        tc_commit(&B->s_full[1]);
-        tc_commit(&B->k_empty[0]);
+        if (leader) {
+          tc_commit(&B->s_full[1]);
+          tc_commit(&B->k_empty[0]);
+        }
       }
       for (int it = 0; it < n_tiles && ok; ++it) {
         const int s = it % kKVStages, s1 = (it + 1) % kKVStages;
         const uint32_t ph = (uint32_t)(it / kKVStages) & 1u, ph1 = (uint32_t)((it + 1) / kKVStages) & 1u;
         const bool more = it + 1 < n_tiles;
-        ok = mbar_wait(&B->v_full[s], ph, B, P.status);
+        ok = wait_all(&B->v_full[s], ph);
         if (!ok) break;
         const uint64_t dv = smem_desc_sw128(smem_u32(sV + s * kTileBytes));
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
-          ok = mbar_wait(&B->p_full[hf], (uint32_t)it & 1u, B, P.status);
+          ok = wait_all(&B->p_full[hf], (uint32_t)it & 1u);
           if (!ok) break;
           tc_fence_after();
+          if (leader) {
 #pragma unroll
-          for (int kk = 0; kk < kHalf / 16; ++kk)   // 16 KV rows = 2048 bytes; P: 8 TMEM columns per 16 bf16
-            mma_ts(tmem + kColO, tmem + kColS + hf * kHalf + kk * 8, dv + (uint64_t)((hf * (kHalf / 16) + kk) * 128),
-                   idesc_pv, (it > 0 || hf > 0 || kk > 0));
-          if (hf == 1) tc_commit(&B->v_empty[s]);
-          if (!more && hf == 0) tc_commit(&B->pv_done);   // (the last half has no later score MMA to tell it by)
+            for (int kk = 0; kk < kHalf / 16; ++kk)   // 16 KV rows = 2048 bytes; P: 8 TMEM columns per 16 bf16
+              mma_ts(tm + kColO, tm + kColS + hf * kHalf + kk * 8, dv + (uint64_t)((hf * (kHalf / 16) + kk) * 128),
+                     idesc_pv, (it > 0 || hf > 0 || kk > 0));
+            if (hf == 1) tc_commit(&B->v_empty[s]);
+            if (!more && hf == 0) tc_commit(&B->pv_done);   // (the last half has no later score MMA to tell it by)
+          }
           if (more) {
             if (hf == 0) {
-              ok = mbar_wait(&B->k_full[s1], ph1, B, P.status);
+              ok = wait_all(&B->k_full[s1], ph1);
               if (!ok) break;
               tc_fence_after();
             }
             issue_qk(s1, hf);
-            tc_commit(&B->s_full[hf]);
-            if (hf == 1) tc_commit(&B->k_empty[s1]);
+            if (leader) {
+              tc_commit(&B->s_full[hf]);
+              if (hf == 1) tc_commit(&B->k_empty[s1]);
+            }
           }
         }
       }
       if (ok) {
-        tc_commit(&B->o_full);
-        mbar_wait(&B->o_full, 0, B, P.status);
+        if (leader) tc_commit(&B->o_full);
+        wait_all(&B->o_full, 0);
       } else {
-        tc_commit(&B->drain);                     // let every issued MMA finish before TMEM is freed
-        mbar_wait(&B->drain, 0, B, P.status);
+        if (leader) tc_commit(&B->drain);           // let every issued MMA finish before TMEM is freed
+        wait_all(&B->drain, 0);
       }
     }
     __syncwarp();
@@ -377,8 +423,8 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (!ok) break;
       tc_fence_after();
       uint32_t s[kHalf];
-      tmem_ld32(t_row + kColS + hf * kHalf, s);
-      tmem_ld32(t_row + kColS + hf * kHalf + 32, s + 32);
+#pragma unroll
+      for (int j = 0; j < kHalf / 32; ++j) tmem_ld32(t_row + kColS + hf * kHalf + j * 32, s + j * 32);
       tmem_wait_ld();
       const int col0 = (t_begin + it) * kBN + hf * kHalf;
       if (col0 + kHalf > P.N) {
@@ -388,12 +434,13 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       // row maximum: four independent chains of 3-input maxima
       float m4[4];
+      constexpr int kChain = kHalf / 4;                  // 24 scores per chain
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        m4[q] = fmaxf(__uint_as_float(s[16 * q]), __uint_as_float(s[16 * q + 1]));
+        m4[q] = fmaxf(__uint_as_float(s[kChain * q]), __uint_as_float(s[kChain * q + 1]));
 #pragma unroll
-        for (int j = 2; j < 16; j += 2)
-          m4[q] = max3(m4[q], __uint_as_float(s[16 * q + j]), __uint_as_float(s[16 * q + j + 1]));
+        for (int j = 2; j < kChain; j += 2)
+          m4[q] = max3(m4[q], __uint_as_float(s[kChain * q + j]), __uint_as_float(s[kChain * q + j + 1]));
       }
       float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * c;
       if (idx == 0) {
@@ -412,14 +459,14 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             mref = mx;
             l *= a;
           }
-          uint32_t o[32];
+          uint32_t o[16];
 #pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            tmem_ld32(t_row + kColO + j * 32, o);
+          for (int j = 0; j < 4; ++j) {
+            tmem_ld16(t_row + kColO + j * 16, o);
             tmem_wait_ld();
 #pragma unroll
-            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * a);
-            tmem_st32(t_row + kColO + j * 32, o);
+            for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * a);
+            tmem_st16(t_row + kColO + j * 16, o);
           }
         }
       }
@@ -437,7 +484,9 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       const float2 t = add2(add2(acc[0], acc[1]), add2(acc[2], acc[3]));
       l += t.x + t.y;
-      tmem_st32(t_row + kColS + hf * kHalf, s);
+      // P: bf16 pairs over the first kHalf / 2 columns of S_hf
+      if constexpr (kHalf / 2 >= 32) tmem_st32(t_row + kColS + hf * kHalf, s);
+      if constexpr ((kHalf / 2) % 32 == 16) tmem_st16(t_row + kColS + hf * kHalf + (kHalf / 64) * 32, s + (kHalf / 64) * 32);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(&B->p_full[hf]);
@@ -545,13 +594,13 @@ inline EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// [rows, C] bf16 row-major; box = 64 columns x 128 rows, 128-byte swizzle, zero fill outside.
-inline int make_rows_map(CUtensorMap* map, const void* base, int rows, int C) {
+// [rows, C] bf16 row-major; box = 64 columns x box_rows rows, 128-byte swizzle, zero fill outside.
+inline int make_rows_map(CUtensorMap* map, const void* base, int rows, int C, int box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return OVGGT_ERR_CUDA;
   cuuint64_t dims[2] = {(cuuint64_t)C, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)C * 2};
-  cuuint32_t box[2] = {kHD, kBN};
+  cuuint32_t box[2] = {(cuuint32_t)kHD, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -566,7 +615,7 @@ inline int make_rows_map(CUtensorMap* map, const void* base, int rows, int C) {
 // Number of KV splits: minimise (waves of CTAs over 2 x 148 slots) x (tiles per CTA + fixed overhead).
 inline int attn_choose_splits(int M, int N, int H) {
   const int q_tiles = (M + kBM - 1) / kBM, tiles = (N + kBN - 1) / kBN;
-  const long slots = 2L * 148;
+  const long slots = (long)kCtasPerSm * 148;
   int best = 1;
   long best_cost = -1;
   for (int s = 1; s <= kMaxSplits && s <= tiles; ++s) {
@@ -575,7 +624,7 @@ inline int attn_choose_splits(int M, int N, int H) {
     if (eff != s) continue;
     const long ctas = (long)q_tiles * H * s;
     const long waves = (ctas + slots - 1) / slots;
-    const long cost = waves * (per + 3) + (s > 1 ? 2 : 0);
+    const long cost = waves * (per + 384 / kBN) + (s > 1 ? 256 / kBN : 0);
     if (best_cost < 0 || cost < best_cost) {
       best_cost = cost;
       best = s;
@@ -596,11 +645,11 @@ inline int attn_tcgen05_launch(const void* q, const void* k, const void* v, int 
                                void* scratch, int* status, cudaStream_t st) {
   const int C = H * kHD;
   CUtensorMap tq, tk, tv;
-  int rc = make_rows_map(&tq, q, M, C);
+  int rc = make_rows_map(&tq, q, M, C, kBM);
   if (rc) return rc;
-  rc = make_rows_map(&tk, k, N, C);
+  rc = make_rows_map(&tk, k, N, C, kBN);
   if (rc) return rc;
-  rc = make_rows_map(&tv, v, N, C);
+  rc = make_rows_map(&tv, v, N, C, kBN);
   if (rc) return rc;
   AttnParams P;
   P.M = M; P.N = N; P.H = H;
