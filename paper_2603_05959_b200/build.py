@@ -1,5 +1,6 @@
 """Build the CUDA library in-tree: paper_2603_05959_b200/libovggt.so (sm_100a only)."""
 import os
+import re
 import subprocess
 import sys
 
@@ -20,16 +21,37 @@ def needs_build() -> bool:
     return any(os.path.getmtime(d) > os.path.getmtime(OUT) for d in deps)
 
 
+def check_register_pool(ptxas_log: str) -> None:
+    """The attention kernel moves registers between its warpgroups with setmaxnreg, inside the pool it was launched
+    with; an increase the pool cannot serve would wait for ever.  The source states the launch count it was budgeted
+    for (kRegsLaunch); refuse a build whose ptxas report says otherwise."""
+    src = open(os.path.join(CSRC, "attn_tcgen05.cuh")).read()
+    want = int(re.search(r"constexpr int kRegsLaunch = (\d+);", src).group(1))
+    m = re.search(r"Compiling entry function '[^']*k_attn_tcgen05[^']*'.*?Used (\d+) registers", ptxas_log, re.S)
+    if not m:
+        raise RuntimeError("ptxas report for k_attn_tcgen05 not found")
+    if int(m.group(1)) != want:
+        raise RuntimeError(f"k_attn_tcgen05 is launched with {m.group(1)} registers, budgeted for {want}")
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not needs_build():
         return OUT
-    cmd = [NVCC, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+    tmp = OUT + ".tmp"
+    cmd = [NVCC, "-Xptxas", "-v", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "--cudart", "static",
-           "-o", OUT, os.path.join(CSRC, "ovggt_api.cu")]
-    if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-    subprocess.run(cmd, check=True)
+           "-o", tmp, os.path.join(CSRC, "ovggt_api.cu")]
+    r = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+    if verbose or r.returncode != 0:
+        print(r.stdout, file=sys.stderr)
+    if r.returncode != 0:
+        raise subprocess.CalledProcessError(r.returncode, cmd)
+    try:
+        check_register_pool(r.stdout)
+    except Exception:
+        os.remove(tmp)
+        raise
+    os.replace(tmp, OUT)
     return OUT
 
 

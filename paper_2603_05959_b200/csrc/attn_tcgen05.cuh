@@ -29,7 +29,11 @@ constexpr int kCtasPerSm = 2;       // resident CTAs per SM
 constexpr int kHD = 64;             // head dim
 constexpr int kKVStages = 2;
 constexpr int kAttnThreads = 256;
-constexpr int kRegsSoftmax = 216, kRegsOther = 40;   // 2 CTAs x (128 x 216 + 128 x 40) = 64K registers
+// setmaxnreg only moves registers inside the pool the CTA was launched with (threads x launch registers), and an
+// increase that the pool cannot serve waits for ever: the two warpgroups must fit 256 x 128.
+constexpr int kRegsLaunch = 128;    // what __launch_bounds__(256, 2) gives: 65536 / 512
+constexpr int kRegsSoftmax = 216, kRegsOther = 40;
+static_assert(128 * kRegsSoftmax + 128 * kRegsOther <= kAttnThreads * kRegsLaunch, "register pool of the CTA exceeded");
 constexpr int kQBytes = kBM * kHD * 2;           // 16 KB
 constexpr int kTileBytes = kBN * kHD * 2;          // 24 KB
 constexpr int kHalf = kBN / 2;      // KV rows per S buffer
