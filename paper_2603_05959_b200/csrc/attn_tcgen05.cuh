@@ -19,6 +19,8 @@
 
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace ovggt {
@@ -40,6 +42,7 @@ constexpr int kHalf = kBN / 2;      // KV rows per S buffer
 constexpr int kTmemCols = 256;
 constexpr int kColS = 0, kColO = 2 * kHalf;   // S_0 at columns [0, 96), S_1 at [96, 192), O at [192, 256): all 256 columns
 constexpr float kRescaleThreshold = 8.0f;          // log2 units
+constexpr int kPolyEvery = 4;                      // one pair of exponentials in kPolyEvery goes to the FMA pipes
 constexpr int kMaxSplits = 16;
 
 struct AttnBarriers {
@@ -221,6 +224,24 @@ __device__ __forceinline__ bool elect_one() {
       "{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(pred));
   return pred != 0;
+}
+// 2^x for a pair on the FMA pipes, for the share of the exponentials taken off the 16-per-clock special-function
+// unit: x = n + f with n = round(x) (magic-number rounding) and f in [-0.5, 0.5], a cubic for 2^f (Chebyshev nodes,
+// relative error 1e-4, below bf16 rounding), and n added into the exponent field.  x is clamped at -125 so that the
+// exponent field cannot wrap; larger x than the rescale threshold only occurs in a pass whose result is discarded.
+__device__ __forceinline__ float2 ex2_poly2(float2 x) {
+  const float kMagic = 12582912.0f;                  // 1.5 * 2^23
+  x.x = fmaxf(x.x, -125.0f);
+  x.y = fmaxf(x.y, -125.0f);
+  const float2 t = add2(x, make_float2(kMagic, kMagic));
+  const float2 n = add2(t, make_float2(-kMagic, -kMagic));
+  const float2 f = fma2(n, make_float2(-1.0f, -1.0f), x);
+  float2 p = fma2(f, make_float2(0.05583828315138817f, 0.05583828315138817f),
+                  make_float2(0.2426394820213318f, 0.2426394820213318f));
+  p = fma2(p, f, make_float2(0.6931367516517639f, 0.6931367516517639f));
+  p = fma2(p, f, make_float2(0.9999245405197144f, 0.9999245405197144f));
+  return make_float2(__int_as_float(__float_as_int(p.x) + (__float_as_int(t.x) << 23)),
+                     __int_as_float(__float_as_int(p.y) + (__float_as_int(t.y) << 23)));
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t d;
@@ -427,29 +448,63 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (!ok) break;
       tc_fence_after();
       uint32_t s[kHalf];
+      auto load_scores = [&]() {
 #pragma unroll
-      for (int j = 0; j < kHalf / 32; ++j) tmem_ld32(t_row + kColS + hf * kHalf + j * 32, s + j * 32);
-      tmem_wait_ld();
-      const int col0 = (t_begin + it) * kBN + hf * kHalf;
-      if (col0 + kHalf > P.N) {
+        for (int j = 0; j < kHalf / 32; ++j) tmem_ld32(t_row + kColS + hf * kHalf + j * 32, s + j * 32);
+        tmem_wait_ld();
+        const int col0 = (t_begin + it) * kBN + hf * kHalf;
+        if (col0 + kHalf > P.N) {
 #pragma unroll
-        for (int j = 0; j < kHalf; ++j)
-          if (col0 + j >= P.N) s[j] = 0xFF800000u;     // -inf on columns past the last row
-      }
-      // row maximum: four independent chains of 3-input maxima
-      float m4[4];
-      constexpr int kChain = kHalf / 4;                  // 24 scores per chain
+          for (int j = 0; j < kHalf; ++j)
+            if (col0 + j >= P.N) s[j] = 0xFF800000u;     // -inf on columns past the last row
+        }
+      };
+      // p = 2^(s * c - mref) on pairs, packed to bf16 over the front of s[]; returns the row's sum of p (four
+      // independent packed partial sums, folded in a fixed order).  With `track` the raw row maximum is gathered in
+      // the same pass (four chains of 3-input maxima), where it hides behind the exponentials.
+      auto exp_pass = [&](auto track, float& raw_max) -> float {
+        const float2 c2 = make_float2(c, c), nm2 = make_float2(-mref, -mref);
+        float2 acc[4];
+        float m4[4];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        m4[q] = fmaxf(__uint_as_float(s[kChain * q]), __uint_as_float(s[kChain * q + 1]));
+        for (int q = 0; q < 4; ++q) {
+          acc[q] = make_float2(0.0f, 0.0f);
+          m4[q] = -INFINITY;
+        }
 #pragma unroll
-        for (int j = 2; j < kChain; j += 2)
-          m4[q] = max3(m4[q], __uint_as_float(s[kChain * q + j]), __uint_as_float(s[kChain * q + j + 1]));
-      }
-      float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * c;
+        for (int j = 0; j < kHalf; j += 2) {
+          const float s0 = __uint_as_float(s[j]), s1 = __uint_as_float(s[j + 1]);
+          if constexpr (decltype(track)::value) m4[(j >> 1) & 3] = max3(m4[(j >> 1) & 3], s0, s1);
+          const float2 x = fma2(make_float2(s0, s1), c2, nm2);
+          const float2 p = ((j >> 1) % kPolyEvery == kPolyEvery - 1) ? ex2_poly2(x) : make_float2(ex2(x.x), ex2(x.y));
+          acc[(j >> 1) & 3] = add2(acc[(j >> 1) & 3], p);
+          s[j >> 1] = pack_bf16(p.x, p.y);
+        }
+        raw_max = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        const float2 t = add2(add2(acc[0], acc[1]), add2(acc[2], acc[3]));
+        return t.x + t.y;
+      };
+      load_scores();
+      float add, raw;
       if (idx == 0) {
-        mref = mx;
+        // the first half fixes the reference: its maximum has to be known before any exponential
+        float m4[4];
+        constexpr int kChain = kHalf / 4;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          m4[q] = fmaxf(__uint_as_float(s[kChain * q]), __uint_as_float(s[kChain * q + 1]));
+#pragma unroll
+          for (int j = 2; j < kChain; j += 2)
+            m4[q] = max3(m4[q], __uint_as_float(s[kChain * q + j]), __uint_as_float(s[kChain * q + j + 1]));
+        }
+        mref = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * c;
+        add = exp_pass(std::false_type{}, raw);
       } else {
+        // Later halves compute p under the reference they inherit while the maximum is gathered, and keep the
+        // result unless the maximum outgrew the reference by more than the threshold (rare); then O is rescaled,
+        // the scores are read again (P has not been written over them yet) and p is recomputed.
+        add = exp_pass(std::true_type{}, raw);
+        const float mx = raw * c;
         const bool grow = mx - mref > kRescaleThreshold;
         if (__any_sync(0xFFFFFFFFu, grow)) {
           // O may still be accumulating the previous half.  PV(idx - 1) is issued just before the scores of half
@@ -472,22 +527,11 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             for (int e = 0; e < 16; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * a);
             tmem_st16(t_row + kColO + j * 16, o);
           }
+          load_scores();
+          add = exp_pass(std::false_type{}, raw);
         }
       }
-      // p = 2^(s * c - mref) on pairs; four independent packed partial sums, folded in a fixed order
-      const float2 c2 = make_float2(c, c), nm2 = make_float2(-mref, -mref);
-      float2 acc[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) acc[q] = make_float2(0.0f, 0.0f);
-#pragma unroll
-      for (int j = 0; j < kHalf; j += 2) {
-        const float2 x = fma2(make_float2(__uint_as_float(s[j]), __uint_as_float(s[j + 1])), c2, nm2);
-        const float2 p = make_float2(ex2(x.x), ex2(x.y));
-        acc[(j >> 1) & 3] = add2(acc[(j >> 1) & 3], p);
-        s[j >> 1] = pack_bf16(p.x, p.y);
-      }
-      const float2 t = add2(add2(acc[0], acc[1]), add2(acc[2], acc[3]));
-      l += t.x + t.y;
+      l += add;
       // P: bf16 pairs over the first kHalf / 2 columns of S_hf
       if constexpr (kHalf / 2 >= 32) tmem_st32(t_row + kColS + hf * kHalf, s);
       if constexpr ((kHalf / 2) % 32 == 16) tmem_st16(t_row + kColS + hf * kHalf + (kHalf / 64) * 32, s + (kHalf / 64) * 32);
