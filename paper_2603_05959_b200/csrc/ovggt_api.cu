@@ -120,7 +120,7 @@ int launch_diversity_from_parts(const void* K, int rows, int C, int dtype, const
   int* arrived = reinterpret_cast<int*>(ksum + C);
   k_colsum_final_sliced<<<dim3((C + 31) / 32, kColsumSlices), 1024, 0, st>>>(part, nparts, C, slices, ksum, arrived);
   LAUNCHED();
-  const int grid = std::min((rows + 15) / 16, 148 * 8);
+  const int grid = std::min((rows + 63) / 64, 148 * 8);   // eight rows per warp: the centroid registers are loaded once
   const size_t smem = (size_t)C * 4;
   const int norm_ctas = resid ? (resid_rows + 7) / 8 : 0;
   if (dtype == kBF16)

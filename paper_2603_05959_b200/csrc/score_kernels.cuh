@@ -153,51 +153,87 @@ __global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, 
     if (row < resid_rows) warp_row_norm<DT>(resid, row, nvec, s_raw);
     return;
   }
-  extern __shared__ float sh_ksum[];
+  extern __shared__ __align__(16) float sh_ksum[];
   const int C = nvec * VEC;
+  const int lane = threadIdx.x & 31;
+  const int warps_total = (int)((div_ctas * (unsigned)blockDim.x) >> 5);
+  // Two rows per iteration, eight 16-byte loads per lane in flight (rows of up to 128 vectors; longer rows loop).
+  // The first pair is requested before the centroid is staged, so that its DRAM latency runs under the set-up.
+  int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5) * 2;
+  uint4 u[2][4];
+  auto load_pair = [&](int r0, int v0) {
+    const uint4* p0 = K + (size_t)r0 * nvec;
+    const uint4* p1 = p0 + (r0 + 1 < rows ? nvec : 0);
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (v0 + 32 * i < nvec) {
+        u[0][i] = ld_nc(p0 + v0 + 32 * i);
+        u[1][i] = ld_nc(p1 + v0 + 32 * i);
+      }
+  };
+  if (row < rows) load_pair(row, lane);
   for (int c = threadIdx.x; c < C; c += blockDim.x) {   // ksum: [n_slices, C], folded in slice order
     float t = ksum[c];
     for (int sl = 1; sl < n_slices; ++sl) t += ksum[(size_t)sl * C + c];
     sh_ksum[c] = t;
   }
   __syncthreads();
-  const int lane = threadIdx.x & 31;
   float kn = 0.0f;
   for (int v = lane; v < nvec; v += 32)
 #pragma unroll
-    for (int e = 0; e < VEC; ++e) kn = __fmaf_rn(sh_ksum[v * VEC + e], sh_ksum[v * VEC + e], kn);
+    for (int e = 0; e < VEC; e += 4) {
+      const float4 k4 = *reinterpret_cast<const float4*>(sh_ksum + v * VEC + e);
+      kn = __fmaf_rn(k4.x, k4.x, kn);
+      kn = __fmaf_rn(k4.y, k4.y, kn);
+      kn = __fmaf_rn(k4.z, k4.z, kn);
+      kn = __fmaf_rn(k4.w, k4.w, kn);
+    }
   kn = warp_sum(kn);
-  const int warps_total = (int)((div_ctas * (unsigned)blockDim.x) >> 5);
-  // two rows per iteration, so that eight 16-byte loads per lane are in flight
-  for (int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5) * 2; row < rows;
-       row += 2 * warps_total) {
+  // A lane meets the same columns in every row; when a row fits one round of loads (nvec <= 128) the lane keeps
+  // its 4 x VEC centroid values in registers, and the row loop does not touch shared memory at all.
+  const bool in_regs = nvec <= 128;
+  float kreg[4][VEC];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int e = 0; e < VEC; e += 4) {
+      float4 k4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+      if (in_regs && lane + 32 * i < nvec) k4 = *reinterpret_cast<const float4*>(sh_ksum + (lane + 32 * i) * VEC + e);
+      kreg[i][e] = k4.x; kreg[i][e + 1] = k4.y; kreg[i][e + 2] = k4.z; kreg[i][e + 3] = k4.w;
+    }
+  for (; row < rows; row += 2 * warps_total) {
     const bool two = row + 1 < rows;
-    const uint4* p0 = K + (size_t)row * nvec;
-    const uint4* p1 = p0 + (two ? nvec : 0);
     float dot[2] = {0.0f, 0.0f}, nrm[2] = {0.0f, 0.0f};
     for (int v0 = lane; v0 < nvec; v0 += 128) {
-      uint4 u[2][4];
+      if (v0 != lane) load_pair(row, v0);
 #pragma unroll
       for (int i = 0; i < 4; ++i)
         if (v0 + 32 * i < nvec) {
-          u[0][i] = ld_nc(p0 + v0 + 32 * i);
-          u[1][i] = ld_nc(p1 + v0 + 32 * i);
-        }
+          float ks[VEC];
+          if (in_regs) {
 #pragma unroll
-      for (int r = 0; r < 2; ++r)
+            for (int e = 0; e < VEC; ++e) ks[e] = kreg[i][e];
+          } else {
+            // 16-byte reads: consecutive lanes are VEC floats apart, which scalar reads would serialise eight ways
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-          if (v0 + 32 * i < nvec) {
+            for (int e = 0; e < VEC; e += 4)
+              *reinterpret_cast<float4*>(ks + e) =
+                  *reinterpret_cast<const float4*>(sh_ksum + (v0 + 32 * i) * VEC + e);
+          }
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
             float f[VEC];
             unpack<DT>(u[r][i], f);
-            const float* ks = sh_ksum + (v0 + 32 * i) * VEC;
 #pragma unroll
             for (int e = 0; e < VEC; ++e) {
               dot[r] = __fmaf_rn(f[e], ks[e], dot[r]);
               nrm[r] = __fmaf_rn(f[e], f[e], nrm[r]);
             }
           }
+        }
     }
+    const int next = row + 2 * warps_total;
+    if (next < rows) load_pair(next, lane);           // the next pair travels during the reductions
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
       const float dt = warp_sum(dot[r]), nr = warp_sum(nrm[r]);
