@@ -38,17 +38,19 @@ __global__ void __launch_bounds__(256) k_compact(const uint4* __restrict__ k_src
 constexpr int kCompactSumMaxVec = 128;   // rows of up to 128 16-byte vectors (C <= 1024 bf16) in the fused variant
 
 // The same gather that also sums, per CTA, the columns of the K rows it writes: part[blockIdx.x, c] = sum of
-// k_dst[j, c] over this CTA's K rows, each warp folding its rows in item order and the CTA folding its four
-// K warps in warp order (the warps of a CTA alternate between K and V items because the total number of warps
-// is even).  The sums over all CTAs are the column sums of the compacted keys: the centroid the next step's
-// diversity score needs, obtained without another pass over K.  Requires nvec <= kCompactSumMaxVec.
+// k_dst[j, c] over this CTA's rows.  A warp takes two survivors per iteration, j and j + (warps in the grid), and
+// moves the K and the V row of both with all 16 loads of a lane issued before the first store: when the kernel
+// shares the SMs with the attention it is the bytes in flight per occupied register that decide how long it holds
+// them.  A warp folds its K rows in the order it meets them; the CTA folds its warps 4..7 onto 0..3 and then 0..3 in
+// order, so the sums do not depend on timing.  The sums over all CTAs are the column sums of the compacted keys: the
+// centroid the next step's diversity score needs, without another pass over K.  Requires nvec <= kCompactSumMaxVec.
 template <int DT>
 __global__ void __launch_bounds__(256) k_compact_colsum(const uint4* __restrict__ k_src, const uint4* __restrict__ v_src,
                                                         const int* __restrict__ survivors, int n_keep, int nvec,
                                                         uint4* __restrict__ k_dst, uint4* __restrict__ v_dst,
                                                         float* __restrict__ part) {
   constexpr int VEC = VecOf<DT>::n;
-  __shared__ float red[4][kCompactSumMaxVec * VEC];
+  __shared__ __align__(16) float red[4][kCompactSumMaxVec * VEC];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
   float acc[4][VEC];
@@ -56,37 +58,56 @@ __global__ void __launch_bounds__(256) k_compact_colsum(const uint4* __restrict_
   for (int i = 0; i < 4; ++i)
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[i][e] = 0.0f;
-  for (int item = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5); item < 2 * n_keep;
-       item += warps_total) {
-    const int j = item >> 1;
-    const int src = survivors[j];
-    if (item & 1) {
-      warp_copy_row(v_src + (size_t)src * nvec, v_dst + (size_t)j * nvec, nvec, lane);
-    } else {
-      const uint4* sp = k_src + (size_t)src * nvec;
-      uint4* dp = k_dst + (size_t)j * nvec;
-      uint4 u[4];
+  for (int j0 = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5); j0 < n_keep; j0 += 2 * warps_total) {
+    const int j1 = j0 + warps_total;
+    const bool two = j1 < n_keep;
+    const int s0 = survivors[j0], s1 = two ? survivors[j1] : s0;
+    const uint4 *ka = k_src + (size_t)s0 * nvec, *va = v_src + (size_t)s0 * nvec;
+    const uint4 *kb = k_src + (size_t)s1 * nvec, *vb = v_src + (size_t)s1 * nvec;
+    uint4 uk[2][4], uv[2][4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (lane + 32 * i < nvec) u[i] = ld_nc(sp + lane + 32 * i);
+    for (int i = 0; i < 4; ++i)
+      if (lane + 32 * i < nvec) {
+        uk[0][i] = ld_nc(ka + lane + 32 * i);
+        uv[0][i] = ld_nc(va + lane + 32 * i);
+        uk[1][i] = ld_nc(kb + lane + 32 * i);
+        uv[1][i] = ld_nc(vb + lane + 32 * i);
+      }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+      if (r == 1 && !two) break;
+      const size_t j = (size_t)(r == 0 ? j0 : j1);
 #pragma unroll
       for (int i = 0; i < 4; ++i)
         if (lane + 32 * i < nvec) {
-          dp[lane + 32 * i] = u[i];
+          k_dst[j * nvec + lane + 32 * i] = uk[r][i];
+          v_dst[j * nvec + lane + 32 * i] = uv[r][i];
           float f[VEC];
-          unpack<DT>(u[i], f);
+          unpack<DT>(uk[r][i], f);
 #pragma unroll
           for (int e = 0; e < VEC; ++e) acc[i][e] += f[e];
         }
     }
   }
-  if ((warp & 1) == 0) {
+  // fold the eight warps: 4..7 park their sums, 0..3 add them to their own and park the result, then four columns-wise
+  auto park = [&](int slot, bool add) {
 #pragma unroll
     for (int i = 0; i < 4; ++i)
       if (lane + 32 * i < nvec)
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) red[warp >> 1][(lane + 32 * i) * VEC + e] = acc[i][e];
-  }
+        for (int e = 0; e < VEC; e += 4) {
+          float4* p = reinterpret_cast<float4*>(&red[slot][(lane + 32 * i) * VEC + e]);
+          float4 t = make_float4(acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]);
+          if (add) {
+            const float4 o = *p;
+            t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
+          }
+          *p = t;
+        }
+  };
+  if (warp >= 4) park(warp - 4, false);
+  __syncthreads();
+  if (warp < 4) park(warp, true);
   __syncthreads();
   const int C = nvec * VEC;
   for (int c = threadIdx.x; c < C; c += blockDim.x)

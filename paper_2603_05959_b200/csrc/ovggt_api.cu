@@ -139,7 +139,7 @@ int launch_compact_colsum(const void* ks, const void* vs, const int* surv, int n
   *nparts = 0;
   if (n_keep <= 0) return OVGGT_OK;
   const int nvec = C * elem_bytes(dtype) / 16;
-  const int grid = std::min((2 * n_keep + 7) / 8, 148 * 8);
+  const int grid = std::min((n_keep + 31) / 32, 148 * 8);   // four survivors (K and V rows) per warp
   if (dtype == kBF16)
     k_compact_colsum<kBF16><<<grid, 256, 0, st>>>((const uint4*)ks, (const uint4*)vs, surv, n_keep, nvec, (uint4*)kd,
                                                   (uint4*)vd, part);
