@@ -347,7 +347,7 @@ def run_ours(args) -> None:
         eb = cfg.elem_bytes
         kernels = {}
         alg_bytes = {"append": 4 * M * C * eb, "row_norms": M * C * eb + 4 * M,
-                     "diversity": 2 * Bud * C * eb + 4 * Bud, "select": 4 * N + N + 4 * Bud,
+                     "diversity": Bud * C * eb + 4 * Bud + M * C * eb + 4 * M, "select": 4 * N + N + 4 * Bud,
                      "compact": 4 * Bud * C * eb}
         for name, rec in prof.items():
             ms = rec["ms"] / max(1, rec["count"])
