@@ -588,6 +588,9 @@ __global__ void __launch_bounds__(256) k_attn_merge(const float* __restrict__ o_
   const int C = H * kHD;
   const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t total = (size_t)M * (C / 4);
+  // launched with programmatic stream serialisation: its CTAs may become resident while the last attention CTAs
+  // drain; the partials are complete and visible once this wait returns
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (idx >= total) return;
   const int m = (int)(idx / (C / 4)), c4 = (int)(idx % (C / 4)), h = (c4 * 4) / kHD;
   float2 ml[kMaxSplits];
@@ -716,8 +719,18 @@ inline int attn_tcgen05_launch(const void* q, const void* k, const void* v, int 
   if (e != cudaSuccess) { g_attn_last_error = (int)e; return OVGGT_ERR_CUDA; }
   if (P.splits > 1) {
     const size_t total = (size_t)M * (C / 4);
-    k_attn_merge<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(P.o_part, P.ml_part, M, H, P.splits, P.out);
-    e = cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((total + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, k_attn_merge, (const float*)P.o_part, (const float2*)P.ml_part, M, H, P.splits, P.out);
+    if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { g_attn_last_error = (int)e; return OVGGT_ERR_CUDA; }
   }
   return OVGGT_OK;
