@@ -130,6 +130,25 @@ def test_attention_bf16_large_logits_exercise_rescaling():
     _attn_check(150, 1500, 2, gen.DTYPE_BF16, 77, qscale=6.0)
 
 
+def test_attention_bf16_scores_rising_along_the_keys():
+    """Keys ordered so that every score half outgrows the running reference maximum by far more than the lazy
+    threshold: each round takes the rescale-and-recompute path, and the softmax concentrates on the last keys."""
+    orc.set_threads(8)
+    M, N, H, dt = 140, 1100, 2, gen.DTYPE_BF16
+    rng = np.random.default_rng(91)
+    u = rng.standard_normal(64).astype(np.float32)
+    u /= np.linalg.norm(u)
+    ramp = (np.arange(N, dtype=np.float32) * 0.25)[:, None]                  # +24 (natural-log units / 8 * 8) per 96 keys
+    k = np.concatenate([ramp * u[None, :] + 0.1 * rng.standard_normal((N, 64)).astype(np.float32) for _ in range(H)], axis=1)
+    q = np.concatenate([(8.0 + rng.random((M, 1)).astype(np.float32)) * u[None, :] for _ in range(H)], axis=1)
+    v = rng.standard_normal((N, H * 64)).astype(np.float32)
+    q, k, v = (gen.round_to_dtype(x, dt) for x in (q, k, v))
+    got = B.k_attention(dev(q, dt), dev(k, dt), dev(v, dt), H).float().cpu().numpy()
+    ref = orc.attention(q, k, v, H, 64)
+    err = np.abs(got - ref)
+    assert np.isfinite(got).all() and err.max() <= ATT_MAX and err.mean() <= ATT_MEAN, (err.max(), err.mean())
+
+
 @pytest.mark.parametrize("M,N,H", [(69, 325, 4), (1, 1, 1), (130, 700, 2)])
 def test_attention_fp32(M, N, H):
     orc.set_threads(8)
