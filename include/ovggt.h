@@ -141,8 +141,9 @@ int ovggt_cache_set_overlap(ovggt_cache* cache, int32_t enable);
  * buffers of the workspace on a copy stream the handle owns (not ordered after earlier work on `stream`), so with
  * pinned host memory the copies of one step overlap the kernels of the step before; the step itself runs on
  * `stream`; out is written by the kernel itself when it is pinned, mapped host memory, and copied back on `stream`
- * otherwise.  The call returns without synchronising: once `stream` has been synchronised, out is valid and the
- * input buffers may be reused. */
+ * otherwise.  When q, k, v and resid lie back to back in that order in host memory they travel as one copy.  The
+ * call returns without synchronising: once `stream` has been synchronised, out is valid and the input buffers may be
+ * reused. */
 int ovggt_layer_step_host(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
 
 /* Counters of one layer.  Synchronises the stream the handle last used (to read the device status word). */

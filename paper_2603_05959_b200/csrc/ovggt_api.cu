@@ -690,10 +690,18 @@ extern "C" int ovggt_layer_step_host(ovggt_cache* h, int32_t layer, const ovggt_
     // the set was last read by the step two calls ago
     if (h->stage_used[p]) CK(cudaStreamWaitEvent(cs, h->ev_done[p], 0));
   }
-  CK(cudaMemcpyAsync(h->stage_q[p], io->q, bytes, cudaMemcpyHostToDevice, cs));
-  CK(cudaMemcpyAsync(h->stage_k[p], io->k, bytes, cudaMemcpyHostToDevice, cs));
-  CK(cudaMemcpyAsync(h->stage_v[p], io->v, bytes, cudaMemcpyHostToDevice, cs));
-  CK(cudaMemcpyAsync(h->stage_r[p], io->resid, bytes, cudaMemcpyHostToDevice, cs));
+  const char* hq = static_cast<const char*>(io->q);
+  const bool packed = static_cast<const char*>(io->k) == hq + bytes && static_cast<const char*>(io->v) == hq + 2 * bytes &&
+                      static_cast<const char*>(io->resid) == hq + 3 * bytes && h->stage_k[p] == h->stage_q[p] + bytes &&
+                      h->stage_v[p] == h->stage_q[p] + 2 * bytes && h->stage_r[p] == h->stage_q[p] + 3 * bytes;
+  if (packed) {   // q | k | v | resid back to back on the host: one copy instead of four
+    CK(cudaMemcpyAsync(h->stage_q[p], io->q, 4 * bytes, cudaMemcpyHostToDevice, cs));
+  } else {
+    CK(cudaMemcpyAsync(h->stage_q[p], io->q, bytes, cudaMemcpyHostToDevice, cs));
+    CK(cudaMemcpyAsync(h->stage_k[p], io->k, bytes, cudaMemcpyHostToDevice, cs));
+    CK(cudaMemcpyAsync(h->stage_v[p], io->v, bytes, cudaMemcpyHostToDevice, cs));
+    CK(cudaMemcpyAsync(h->stage_r[p], io->resid, bytes, cudaMemcpyHostToDevice, cs));
+  }
   if (io->conf) CK(cudaMemcpyAsync(h->stage_conf[p], io->conf, (size_t)h->Np * 4, cudaMemcpyHostToDevice, cs));
   if (h->copy) {
     CK(cudaEventRecord(h->ev_h2d[p], cs));

@@ -22,10 +22,18 @@ class DeviceFrame:
     def __init__(self, cfg: gen.StreamConfig, fi: gen.FrameInputs, device=None, pin: bool = False):
         self.frame_id = fi.frame_id
         self.rho = fi.rho
-        self.q = to_torch(fi.q, cfg.dtype, device, pin)
-        self.k = to_torch(fi.k, cfg.dtype, device, pin)
-        self.v = to_torch(fi.v, cfg.dtype, device, pin)
-        self.resid = to_torch(fi.resid, cfg.dtype, device, pin)
+        if device is None and pin:
+            # one pinned block [q | k | v | resid]: the host-buffer entry point then moves it with a single copy
+            block = torch.empty((4,) + fi.q.shape, dtype=torch_dtype(cfg.dtype)).pin_memory()
+            for i, x in enumerate((fi.q, fi.k, fi.v, fi.resid)):
+                block[i].copy_(to_torch(x, cfg.dtype))
+            self.block = block
+            self.q, self.k, self.v, self.resid = block[0], block[1], block[2], block[3]
+        else:
+            self.q = to_torch(fi.q, cfg.dtype, device, pin)
+            self.k = to_torch(fi.k, cfg.dtype, device, pin)
+            self.v = to_torch(fi.v, cfg.dtype, device, pin)
+            self.resid = to_torch(fi.resid, cfg.dtype, device, pin)
         conf = torch.from_numpy(fi.conf)
         self.conf = conf.to(device) if device is not None else (conf.pin_memory() if pin else conf)
 
