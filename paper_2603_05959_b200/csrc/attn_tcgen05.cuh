@@ -1,18 +1,21 @@
 // bf16 flash attention for sm_100a: out = softmax(Q K^T / sqrt(64)) V per head, head_dim 64, no mask.
 //
-// One CTA owns one 128-row query tile of one head and a contiguous range of 128-row KV tiles.  Each KV
-// tile is processed as two 64-row halves with their own S buffer in tensor memory, so the MMAs of one half
+// One CTA owns one 128-row query tile of one head and a contiguous range of 192-row KV tiles.  Each KV
+// tile is processed as two 96-row halves with their own S buffer in tensor memory, so the MMAs of one half
 // run while the softmax warps work on the other and the softmax never waits for a whole QK^T -> PV chain.
-//   warps 0-3   softmax: one thread per query row reads its 64 S values of a half with tcgen05.ld, keeps a
-//               running reference maximum (rescaling O only when the maximum grows by more than 2^8),
-//               writes P as bf16 over the first 32 columns of that half, and at the end normalises and stores O
+//   warps 0-3   softmax: one thread per query row reads its 96 S values of a half with tcgen05.ld, keeps a
+//               running reference maximum (rescaling O only when the maximum grows by more than 2^8; the maximum
+//               is gathered inside the exponential pass, and the pass is repeated in the rare case that it outgrew
+//               the reference), takes one pair of exponentials in four on the FMA pipes, writes P as bf16 over the
+//               first 48 columns of that half, and at the end normalises and stores O
 //   warp 4      TMA producer: Q once, then K and V tiles into 128-byte-swizzled shared-memory stages
 //   warp 5      allocates tensor memory and issues tcgen05.mma:  S_h = Q K_h^T  (SS, fp32 in TMEM),
-//               O += P_h V_h (P read from TMEM as the A operand, V MN-major from shared memory)
+//               O += P_h V_h (P read from TMEM as the A operand, V MN-major from shared memory); the whole warp
+//               walks the loop so that descriptors stay warp-uniform, one elected lane issues
 //   warps 6-7   only complete the second warpgroup, which hands its registers to the softmax warpgroup
 // With head_dim 64 a 128 x 128 tile needs 512 tensor-pipe cycles but 1024 cycles of the 16-per-clock
-// exponential unit, so the exponentials bound the kernel; two CTAs are resident per SM (256 TMEM columns and
-// ~82 KB shared memory each) to keep that unit fed from two independent query tiles.  The KV range may be split
+// exponential unit, so the softmax rounds bound the kernel; two CTAs are resident per SM (256 TMEM columns and
+// ~115 KB shared memory each) to keep that unit fed from two independent query tiles.  The KV range may be split
 // across CTAs; partial (O, max, sum) triples are merged by a second kernel.  Every mbarrier wait is bounded: on
 // expiry the CTA records OVGGT_ERR_TIMEOUT in the status word and leaves through the common teardown.
 #pragma once

@@ -137,7 +137,8 @@ __global__ void __launch_bounds__(1024) k_colsum_final_sliced(const float* __res
 }
 
 // d[row] = 1 - (k_row . ksum) / (|k_row| |ksum|); the cosine with the centroid equals the cosine
-// with the column sum.  A zero vector has cosine 0.  One warp per row, ksum staged in shared memory;
+// with the column sum.  A zero vector has cosine 0.  One warp per pair of rows; ksum is staged in shared memory
+// once per CTA and, for rows of up to 128 vectors, kept in registers by the lanes that meet its columns;
 // |ksum|^2 is folded by every warp in the same order, so all CTAs agree on it.
 template <int DT>
 __global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, int rows, int nvec,
