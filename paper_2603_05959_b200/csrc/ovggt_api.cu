@@ -588,7 +588,7 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
   P.r_out = S.r; P.survivors = S.surv;
   P.status = h->status; P.n_keep_out = S.n_keep_dev;
   const int ncta = select_cluster_ctas(N);
-  const size_t smem = select_smem_bytes((N + ncta - 1) / ncta, h->Np);
+  const size_t smem = compress_smem_bytes((N + ncta - 1) / ncta, h->Np, M);
   if (smem > kSmemLimit) return OVGGT_ERR_UNSUPPORTED;
   CK(cudaFuncSetAttribute(k_compress_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit));
   {

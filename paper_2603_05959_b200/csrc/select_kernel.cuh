@@ -232,6 +232,13 @@ __host__ __device__ inline size_t select_smem_bytes(int span, int np) {
          (size_t)np * 4 + (((size_t)np + 15) & ~(size_t)15) + 16;
 }
 
+// The fused per-step kernel also keeps the ids and stored scores of its positions (12 bytes each) and the frame's
+// raw residual norms (m floats) on chip.
+__host__ __device__ inline size_t compress_smem_bytes(int span, int np, int m) {
+  return select_smem_bytes(span, np) + (((size_t)span * 8 + 15) & ~(size_t)15) + (((size_t)span * 4 + 15) & ~(size_t)15) +
+         (((size_t)m * 4 + 15) & ~(size_t)15) + 16;
+}
+
 // ---- standalone selection over given priorities: one cluster per independent problem (blockIdx.y)
 
 __global__ void __launch_bounds__(kSelectThreads) k_select(const float* __restrict__ r,
@@ -275,7 +282,7 @@ struct CompressParams {
   const float* d;                   // [n] key diversity (hybrid mode)
   const float* conf;                // [grid_h*grid_w]
   const float* override_r;          // [N] or nullptr
-  const long long* ids_src; const uint8_t* flags_src; float* stored_src;         // [N] pre-compaction meta (stored: new rows filled here)
+  const long long* ids_src; const uint8_t* flags_src; const float* stored_src;   // [N] pre-compaction meta
   long long* ids_dst; uint8_t* flags_dst; float* stored_dst;                     // [<=B] compacted meta
   float* r_out;                     // [N] priorities as computed here
   int* survivors;                   // [min(N, B)]
@@ -283,12 +290,12 @@ struct CompressParams {
   int* n_keep_out;
 };
 
-// Eq. 6 for new-frame token j (aux tokens keep their raw score).
-__device__ __forceinline__ float smoothed_score(const CompressParams& P, int j) {
-  float v = P.s_raw[j];
+// Eq. 6 for new-frame token j (aux tokens keep their raw score); s_raw: the frame's M residual norms.
+__device__ __forceinline__ float smoothed_score(const CompressParams& P, const float* s_raw, int j) {
+  float v = s_raw[j];
   if (j >= P.n_special) {
     const int q = j - P.n_special, y = q / P.grid_w, x = q - y * P.grid_w;
-    const float* S = P.s_raw + P.n_special;
+    const float* S = s_raw + P.n_special;
     float conv = 0.0f;
 #pragma unroll
     for (int dy = -1; dy <= 1; ++dy)
@@ -320,6 +327,10 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
   uint8_t* keep = fl + span16;                             // [span]
   uint32_t* ckeys = reinterpret_cast<uint32_t*>(keep + span16);   // [Np] confidence keys
   uint8_t* cmark = reinterpret_cast<uint8_t*>(ckeys + Np);        // [Np]
+  unsigned char* q8 = smem + ((select_smem_bytes(span, Np) + 15) & ~(size_t)15);
+  long long* sid = reinterpret_cast<long long*>(q8);              // [span] ids of the owned positions
+  float* sst = reinterpret_cast<float*>(q8 + (((size_t)span * 8 + 15) & ~(size_t)15));   // [span] their stored scores
+  float* sraw = sst + (((size_t)span + 3) & ~(size_t)3);          // [M] the frame's residual norms
 
   // -- anchor registration (Sec. 3.3): the A most confident patch tokens of the new frame, ties to the lower
   //    index.  Every CTA computes the same marks and uses those of the positions it owns.
@@ -330,23 +341,51 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
     block_top_mark(ckeys, cmark, Np, P.A, sh);
   }
 
-  // -- protection flags and values of the owned positions
-  for (int i = tid; i < cnt; i += nthr) {
-    const int g = begin + i;
-    uint8_t f = P.flags_src[g] & 3;
-    float x;
-    if (g >= n) {
-      const int j = g - n;
-      if (P.protect_new) f = OVGGT_FLAG_INIT;
-      if (reg && j >= P.n_special && cmark[j - P.n_special]) f = OVGGT_FLAG_HIST;
-      x = smoothed_score(P, j);
-      P.stored_src[g] = x;       // the score the row keeps (read back below by the same CTA when the row survives)
-    } else {
-      if (P.demote_frame >= 0 && f == OVGGT_FLAG_HIST && P.ids_src[g] / M == P.demote_frame) f = OVGGT_FLAG_EVICTABLE;
-      x = (P.mode == OVGGT_SCORE_HYBRID) ? P.d[g] : P.stored_src[g];
+  // -- protection flags and values of the owned positions.  A CTA that owns new rows first stages the frame's raw
+  //    norms (Eq. 6 reads each nine times); all global loads of four positions are issued before any is used.
+  if (end > n) {
+    for (int j = tid; j < M; j += nthr) sraw[j] = P.s_raw[j];
+    __syncthreads();
+  }
+  for (int i0 = tid; i0 < cnt; i0 += 4 * nthr) {
+    uint8_t f4[4];
+    long long id4[4];
+    float d4[4], st4[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * nthr, g = begin + i;
+      if (i < cnt) {
+        f4[u] = P.flags_src[g];
+        id4[u] = P.ids_src[g];
+        if (g < n) {
+          st4[u] = P.stored_src[g];
+          d4[u] = (P.mode == OVGGT_SCORE_HYBRID) ? P.d[g] : 0.0f;
+        }
+      }
     }
-    fl[i] = f;
-    val[i] = x;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * nthr, g = begin + i;
+      if (i < cnt) {
+        uint8_t f = f4[u] & 3;
+        float x, keepscore;
+        if (g >= n) {
+          const int j = g - n;
+          if (P.protect_new) f = OVGGT_FLAG_INIT;
+          if (reg && j >= P.n_special && cmark[j - P.n_special]) f = OVGGT_FLAG_HIST;
+          x = smoothed_score(P, sraw, j);
+          keepscore = x;           // the score the row keeps
+        } else {
+          if (P.demote_frame >= 0 && f == OVGGT_FLAG_HIST && id4[u] / M == P.demote_frame) f = OVGGT_FLAG_EVICTABLE;
+          x = (P.mode == OVGGT_SCORE_HYBRID) ? d4[u] : st4[u];
+          keepscore = st4[u];
+        }
+        fl[i] = f;
+        val[i] = x;
+        sid[i] = id4[u];
+        sst[i] = keepscore;
+      }
+    }
   }
   __syncthreads();
 
@@ -419,11 +458,10 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
     int j = my_base + block_excl_scan_int(c, sh->scan, &tot);
     for (int i = lo; i < hi; ++i)
       if (keep[i]) {
-        const int g = begin + i;
         if (j < P.B) {
-          P.ids_dst[j] = P.ids_src[g];
+          P.ids_dst[j] = sid[i];
           P.flags_dst[j] = fl[i];
-          P.stored_dst[j] = P.stored_src[g];
+          P.stored_dst[j] = sst[i];
         }
         ++j;
       }
