@@ -95,3 +95,23 @@ def test_null_handle_and_strerror(lib):
     assert lib.ovggt_kernel_launches() == 0
     assert lib.ovggt_k_row_norms(None, 1, 64, 0, None, None) == -1
     assert lib.ovggt_k_select(None, None, 0, 0, 1, None, None, None) == -1
+
+
+def test_build_refuses_an_attention_kernel_with_another_launch_register_count():
+    """setmaxnreg moves registers inside the pool the CTA is launched with; the build checks ptxas' launch count
+    against the count the warpgroup budgets in the source were written for."""
+    import re
+    from paper_2603_05959_b200 import build as bld
+    src = open(os.path.join(bld.CSRC, "attn_tcgen05.cuh")).read()
+    want = int(re.search(r"constexpr int kRegsLaunch = (\d+);", src).group(1))
+    soft = int(re.search(r"constexpr int kRegsSoftmax = (\d+), kRegsOther = (\d+);", src).group(1))
+    other = int(re.search(r"constexpr int kRegsSoftmax = (\d+), kRegsOther = (\d+);", src).group(2))
+    threads = int(re.search(r"constexpr int kAttnThreads = (\d+);", src).group(1))
+    assert threads == 256 and 128 * soft + 128 * other <= threads * want        # the pool rule itself
+    log = ("ptxas info    : Compiling entry function '_ZN5ovggt14k_attn_tcgen05E14CUtensorMap_stS0_S0_NS_10AttnParamsE' "
+           "for 'sm_100a'\nptxas info    : Function properties\nptxas info    : Used %d registers, used 1 barriers\n")
+    bld.check_register_pool(log % want)
+    with pytest.raises(RuntimeError):
+        bld.check_register_pool(log % (want - 8))
+    with pytest.raises(RuntimeError):
+        bld.check_register_pool("ptxas info    : nothing about that kernel\n")
