@@ -7,6 +7,8 @@ from oracle import oracle as orc
 from paper_2603_05959_b200 import binding as B
 from paper_2603_05959_b200 import inputs as gen
 
+from attn_cases import assert_attention_close_relative, sampled_rows_all_groups, tiled_hot_case
+
 pytestmark = pytest.mark.gpu
 
 # Tolerances (derived from the arithmetic):
@@ -163,6 +165,35 @@ def test_attention_bf16_full_size_sampled_rows():
     got = _attn_check(1374, 17758, 16, gen.DTYPE_BF16, 30, rows=rows)
     # properties that hold at any size: finite, and each output inside the range of V per column
     assert np.abs(got).max() < 6.0
+
+
+def test_attention_bf16_full_size_peaked_logits_every_key_block_matters():
+    """The bench shape again (5 KV splits x 19 tiles, 94-row tail, ragged last query tile) on data that can fail it:
+    see tiled_hot_case.  As a self-check of the data, the reference is recomputed without the last key block and
+    without the middle fifth of the keys and must then violate the criterion the kernel has to meet."""
+    orc.set_threads(max(1, min(32, torch.get_num_threads())))
+    M, N, H = 1374, 17758, 16
+    q, k, v = tiled_hot_case(M, N, H, 41)
+    rows = sampled_rows_all_groups(M)
+    assert len(rows) >= 24 and rows.max() >= 1280
+    got = B.k_attention(dev(q, 1), dev(k, 1), dev(v, 1), H).float().cpu().numpy()
+    assert np.isfinite(got).all()
+    ref = orc.attention(q, k, v, H, 64, rows=rows)
+    assert_attention_close_relative(got[rows], ref, "bench shape, peaked")
+    for lo, hi in ((92 * 192, N), (7104, 10752)):            # the ragged last block; KV tiles 37..55 (the middle split)
+        keep = np.r_[0:lo, hi:N]
+        broken = orc.attention(q, k[keep], v[keep], H, 64, rows=rows)
+        with pytest.raises(AssertionError):
+            assert_attention_close_relative(broken, ref)
+
+
+@pytest.mark.parametrize("M,N,H", [(300, 2500, 2), (1041, 13329, 2)])
+def test_attention_bf16_peaked_logits_other_shapes(M, N, H):
+    orc.set_threads(max(1, min(32, torch.get_num_threads())))
+    q, k, v = tiled_hot_case(M, N, H, 43 + M)
+    rows = sampled_rows_all_groups(M)
+    got = B.k_attention(dev(q, 1), dev(k, 1), dev(v, 1), H).float().cpu().numpy()
+    assert_attention_close_relative(got[rows], orc.attention(q, k, v, H, 64, rows=rows), f"{M}x{N}")
 
 
 def test_attention_is_deterministic():

@@ -12,6 +12,8 @@ from paper_2603_05959_b200 import binding as B
 from paper_2603_05959_b200 import inputs as gen
 from paper_2603_05959_b200.stream import DeviceFrame, out_to_f32, storage_to_f32
 
+from attn_cases import assert_attention_close_relative, sampled_rows_all_groups, tiled_hot_case
+
 pytestmark = pytest.mark.gpu
 
 R_ATOL = 2e-5          # priorities live in [0, 0.5]; fp32 scores after min-max against fp64
@@ -248,4 +250,32 @@ def test_config2_full_size_through_layer_step_with_overlap():
     assert np.array_equal(storage_to_f32(ex["k"], cfg.dtype), rx["k"])
     assert np.array_equal(storage_to_f32(ex["v"], cfg.dtype), rx["v"])
     assert cache.stats(0)["device_status"] == 0
+    cache.destroy()
+
+
+def test_layer_step_at_steady_state_on_peaked_logits_every_key_block_matters():
+    """ovggt_layer_step at the benchmark's steady state (N = B + M = 17758 rows, overlap on) with keys and values
+    whose every 192-row block carries weight for some query rows (see attn_cases.tiled_hot_case): the cache is
+    imported with the first B rows, the frame brings the last M, and the attention output is compared on rows of
+    every group, rows of the ragged last query tile included."""
+    cfg = gen.config_vggt_layer()
+    orc.set_threads(max(1, min(32, torch.get_num_threads())))
+    M, Bud, H = cfg.tokens_per_frame, cfg.budget, cfg.n_heads
+    N = Bud + M
+    q, k, v = tiled_hot_case(M, N, H, 47)
+    rows = sampled_rows_all_groups(M, seed=9)
+    cache = B.OvggtCache.from_stream(cfg)
+    flags = np.zeros(Bud, np.uint8)
+    flags[:M] = B.FLAG_INIT
+    t_next = -(-Bud // M)
+    cache.import_(0, np.arange(Bud, dtype=np.int64), flags, np.ones(Bud, np.float32), gen.bf16_round_bits(k[:Bud]),
+                  gen.bf16_round_bits(v[:Bud]), next_frame_id=t_next, last_registration_frame=0)
+    fi = gen.frame_inputs(cfg, t_next, fields=("resid",))
+    to = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16).cuda()
+    out = cache.layer_step(0, t_next, to(q), to(k[Bud:]), to(v[Bud:]), to(fi.resid), torch.from_numpy(fi.conf).cuda(), fi.rho)
+    got = out_to_f32(out)
+    assert np.isfinite(got).all()
+    assert_attention_close_relative(got[rows], orc.attention(q, k, v, H, 64, rows=rows), "layer_step, steady state")
+    st = cache.stats(0)
+    assert st["device_status"] == 0 and st["n_cached"] == Bud and st["last_n_candidates"] == N
     cache.destroy()

@@ -384,6 +384,50 @@ def test_score_override_and_stored_mode():
     assert np.all(ex["stored"] > 0)
 
 
+def test_stored_scores_travel_with_their_rows_through_every_compaction():
+    """Stored-residual reading of the score (Sec. 3.2, Activation Value Rating + smoothing): a cached row ranks by
+    the smoothed norm it received in the frame that brought it in.  That value has to move with the row every time
+    the cache is compacted.  Expected values are rebuilt here per token id from each frame's own residual (numpy
+    norm, scipy Gaussian for the interior of the map) and compared, after several evictions, with what the oracle
+    exports and with the priorities it ranks the historical rows by."""
+    cfg = gen.config_tiny().replace(score_mode=gen.SCORE_RESIDUAL_STORED, budget=150, anchor_tokens=4,
+                                    min_anchor_interval=3, tau=0.9)
+    layer = orc.OracleLayer.from_stream(cfg)
+    M, ns, gh, gw = cfg.tokens_per_frame, cfg.n_special, cfg.grid_h, cfg.grid_w
+    expected = {}                                             # token id -> fp32 score it was given when new
+    evictions = 0
+    for t in range(9):
+        fi = gen.frame_inputs(cfg, t)
+        s = np.linalg.norm(fi.resid.astype(np.float64), axis=1)
+        sm = orc.smooth(s, ns, gh, gw, cfg.alpha)
+        # the interior of the patch map against a library Gaussian (3x3, sigma 1 == truncate 1)
+        lib_map = scipy.ndimage.gaussian_filter(s[ns:].reshape(gh, gw), sigma=1.0, truncate=1.0, mode="nearest")
+        np.testing.assert_allclose(sm[ns:].reshape(gh, gw), cfg.alpha * lib_map + (1 - cfg.alpha) * s[ns:].reshape(gh, gw),
+                                   rtol=1e-12)
+        for j in range(M):
+            expected[t * M + j] = np.float32(sm[j])
+        layer.attend(t, fi.q, fi.k, fi.v, compute=False)
+        pre = layer.export(with_kv=False)                     # pre-compaction ids and flags (new rows appended)
+        out = layer.compress(fi.resid, fi.conf, fi.rho)
+        n = len(pre["ids"]) - M
+        evictions += len(pre["ids"]) - len(out["survivors"]) > 0
+        # historical evictable rows rank by the value they were given when new, whatever moved in between
+        hist = [i for i in range(n) if np.isfinite(out["r"][i])]
+        assert all(out["r"][i] == expected[int(pre["ids"][i])] for i in hist), t
+        if t > 2:
+            assert len(hist) > 0
+        # new rows rank by this frame's smoothed norms
+        newfin = [j for j in range(M) if np.isfinite(out["r"][n + j])]
+        assert all(out["r"][n + j] == np.float32(sm[j]) for j in newfin)
+        # and every survivor carries its own value, not a neighbour's
+        ex = layer.export(with_kv=False)
+        want = np.array([expected[int(i)] for i in ex["ids"]], dtype=np.float32)
+        np.testing.assert_array_equal(ex["stored"], want, err_msg=f"frame {t}")
+    assert evictions >= 5                                     # the carry was exercised repeatedly
+    # rows of several different frames are still present, so a carry error could not hide behind a single frame
+    assert len({int(i) // M for i in layer.export(with_kv=False)["ids"]}) >= 3
+
+
 def test_create_rejects_budget_below_protected_bound():
     with pytest.raises(ValueError):
         _tiny_layer(budget=14 + 2 * 3 - 1)          # M + K_max * A = 20
