@@ -108,9 +108,11 @@ typedef struct {
  * cfg->workspace / workspace_bytes are ignored here. */
 size_t ovggt_workspace_bytes(const ovggt_config* cfg);
 
-/* Validate cfg, lay the caches out in cfg->workspace and return a handle.  Enqueues one
- * small clearing kernel on the legacy default stream and synchronises it.
- * OVGGT_ERR_BUDGET_TOO_SMALL if a layer's budget cannot hold the protected set (Eq. 9). */
+/* Validate cfg, lay the caches out in cfg->workspace and return a handle.  Clears a few words of the
+ * workspace on the legacy default stream and synchronises.
+ * OVGGT_ERR_BUDGET_TOO_SMALL if a layer's budget cannot hold the protected set (Eq. 9).
+ * OVGGT_ERR_UNSUPPORTED if a layer's B + M candidates do not fit the selection kernel, which keeps them in the
+ * shared memory of one 8-CTA cluster (about 18 bytes per candidate and CTA: B + M up to roughly 90,000). */
 int ovggt_cache_create(const ovggt_config* cfg, ovggt_cache** out);
 int ovggt_cache_destroy(ovggt_cache* cache);
 
@@ -122,7 +124,9 @@ int ovggt_layer_attend(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* 
 /* Eq. 5-8 and Sec. 3.3 for the frame appended by the last ovggt_layer_attend of this layer:
  * score, protect, select the survivors and compact the cache to <= B^(l) rows, order preserved.
  * The anchor decision of a frame is taken once (first layer that compresses it) from rho and the
- * interval rule and applied identically to every layer.  Uses frame_id, resid, conf, rho,
+ * interval rule and applied identically to every layer.  The anchor state belongs to the handle and only moves
+ * forward: every layer has to compress frame t before any layer compresses a later frame; a layer that comes
+ * with an older frame gets OVGGT_ERR_FRAME_ORDER and nothing is changed.  Uses frame_id, resid, conf, rho,
  * score_override. */
 int ovggt_layer_compress(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
 
@@ -155,12 +159,19 @@ int ovggt_cache_stats(ovggt_cache* cache, int32_t layer, ovggt_stats* out);
 int ovggt_cache_export(ovggt_cache* cache, int32_t layer, int64_t* token_ids, uint8_t* flags,
                        float* scores, void* k, void* v, int32_t* n);
 
-/* Replace the layer's content by n rows given as host arrays (ascending token ids).  Anchor bookkeeping is
- * rebuilt from the flags and ids; next_frame_id is the smallest frame id the stream may continue with.
- * Synchronises. */
+/* Replace the layer's content by n rows given as host arrays (ascending token ids); next_frame_id is the
+ * smallest frame id the stream may continue with.  The per-layer counters are rebuilt from the flags and ids.
+ * The anchor FIFO, the first frame and the last registration belong to the whole handle: a handle that has seen
+ * no frame adopts them from the first non-empty layer imported (FIFO = the frames of its HIST rows, oldest first;
+ * first frame = its first row's frame; last_registration_frame as given); every later non-empty import must agree
+ * with them (OVGGT_ERR_INVALID_ARG otherwise, nothing changed); an empty import never touches them.  To load a
+ * different stream into a used handle, call ovggt_cache_reset first.  Synchronises. */
 int ovggt_cache_import(ovggt_cache* cache, int32_t layer, const int64_t* token_ids, const uint8_t* flags,
                        const float* scores, const void* k, const void* v, int32_t n,
                        int64_t next_frame_id, int64_t last_registration_frame);
+
+/* Forget every frame: all layers empty, no anchors, no first frame, device status cleared.  Synchronises. */
+int ovggt_cache_reset(ovggt_cache* cache);
 
 /* Results of the layer's last compress, copied to host (each pointer may be NULL): priorities [N] as the
  * library computed them (+inf on protected rows; its own values even when score_override was ranked instead),

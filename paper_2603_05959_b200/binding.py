@@ -24,7 +24,7 @@ PROF_CLASSES = ["append", "attention", "row_norms", "diversity", "select", "comp
 EXPORTED = [
     "ovggt_workspace_bytes", "ovggt_cache_create", "ovggt_cache_destroy", "ovggt_layer_attend",
     "ovggt_layer_compress", "ovggt_layer_step", "ovggt_layer_step_host", "ovggt_cache_stats",
-    "ovggt_cache_export", "ovggt_cache_import", "ovggt_cache_last_selection", "ovggt_kernel_launches",
+    "ovggt_cache_export", "ovggt_cache_import", "ovggt_cache_reset", "ovggt_cache_last_selection", "ovggt_kernel_launches",
     "ovggt_cache_profile_enable", "ovggt_cache_profile_read", "ovggt_cache_set_overlap",
     "ovggt_strerror", "ovggt_last_cuda_error", "ovggt_k_row_norms", "ovggt_k_diversity_scratch_bytes",
     "ovggt_k_diversity", "ovggt_k_diversity_static", "ovggt_k_select", "ovggt_k_compact", "ovggt_k_attention_scratch_bytes",
@@ -91,6 +91,7 @@ def lib():
         L.ovggt_cache_stats.argtypes = [vp, i32, C.POINTER(OvggtStats)]
         L.ovggt_cache_export.argtypes = [vp, i32, vp, vp, vp, vp, vp, C.POINTER(i32)]
         L.ovggt_cache_import.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32, i64, i64]
+        L.ovggt_cache_reset.argtypes = [vp]
         L.ovggt_cache_last_selection.argtypes = [vp, i32, vp, C.POINTER(i32), vp, C.POINTER(i32)]
         L.ovggt_cache_profile_enable.argtypes = [vp, i32]
         L.ovggt_cache_set_overlap.argtypes = [vp, i32]
@@ -259,6 +260,9 @@ class OvggtCache:
         _check(lib().ovggt_cache_import(self._h, layer, ids.ctypes.data, flags.ctypes.data, scores.ctypes.data,
                                         k.ctypes.data, v.ctypes.data, len(ids), int(next_frame_id),
                                         int(last_registration_frame)), "ovggt_cache_import")
+
+    def reset(self) -> None:
+        _check(lib().ovggt_cache_reset(self._h), "ovggt_cache_reset")
 
     def set_overlap(self, on: bool) -> None:
         _check(lib().ovggt_cache_set_overlap(self._h, int(on)), "ovggt_cache_set_overlap")

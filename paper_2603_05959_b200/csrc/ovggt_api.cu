@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdio>
@@ -291,6 +292,12 @@ bool config_ok(const ovggt_config* c, int* err) {
       return false;
     }
     if ((int64_t)c->budget[l] + M > (1 << 30)) return false;
+    // the fused selection kernel keeps all B + M candidates of a layer in the shared memory of one cluster
+    const int N = c->budget[l] + (int)M, ncta = select_cluster_ctas(N);
+    if (compress_smem_bytes((N + ncta - 1) / ncta, c->grid_h * c->grid_w, (int)M) > kSmemLimit) {
+      *err = OVGGT_ERR_UNSUPPORTED;
+      return false;
+    }
   }
   *err = OVGGT_OK;
   return true;
@@ -534,7 +541,15 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
   const int M = h->M, C = h->C, n = S.n, N = n + M, B = S.budget, b = S.cur;
   const int64_t t = io->frame_id;
 
-  // Anchor decision of this frame (Sec. 3.3), taken once and shared by all layers.
+  const int ncta = select_cluster_ctas(N);
+  const size_t smem = compress_smem_bytes((N + ncta - 1) / ncta, h->Np, M);
+  if (smem > kSmemLimit) return OVGGT_ERR_UNSUPPORTED;   // (create already refuses such budgets)
+  // The anchor state belongs to the whole handle and moves forward only: a layer that comes with a frame older
+  // than the last decision would take that frame's decision a second time.
+  if (t < h->decided_frame) return OVGGT_ERR_FRAME_ORDER;
+
+  // Anchor decision of this frame (Sec. 3.3), taken once and shared by all layers; nothing below can fail on
+  // an argument any more.
   if (h->decided_frame != t) {
     h->decided_frame = t;
     h->decided_register = false;
@@ -587,9 +602,6 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
   P.ids_dst = S.ids[b ^ 1]; P.flags_dst = S.flags[b ^ 1]; P.stored_dst = S.stored[b ^ 1];
   P.r_out = S.r; P.survivors = S.surv;
   P.status = h->status; P.n_keep_out = S.n_keep_dev;
-  const int ncta = select_cluster_ctas(N);
-  const size_t smem = compress_smem_bytes((N + ncta - 1) / ncta, h->Np, M);
-  if (smem > kSmemLimit) return OVGGT_ERR_UNSUPPORTED;
   CK(cudaFuncSetAttribute(k_compress_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit));
   {
     ProfScope ps(h, OVGGT_PROF_SELECT, st);
@@ -800,6 +812,17 @@ extern "C" int ovggt_cache_import(ovggt_cache* h, int32_t layer, const int64_t* 
     } else if (flags[i] != OVGGT_FLAG_EVICTABLE) return OVGGT_ERR_INVALID_ARG;
   }
   if ((int)anchor_frames.size() > h->cfg.k_max) return OVGGT_ERR_INVALID_ARG;
+  // The anchor FIFO, the first frame and the last registration belong to the handle, not to a layer.  A handle that
+  // has seen no frame adopts them from the first non-empty layer imported; every later import has to agree.
+  const bool fresh = h->first_frame < 0;
+  if (n > 0 && !fresh) {
+    const int64_t f0 = token_ids[0] / M;
+    if (h->cfg.protect_first_frame ? f0 != h->first_frame : f0 < h->first_frame) return OVGGT_ERR_INVALID_ARG;
+    if (anchor_frames.size() != h->anchors.size() ||
+        !std::equal(anchor_frames.begin(), anchor_frames.end(), h->anchors.begin()))
+      return OVGGT_ERR_INVALID_ARG;
+    if (last_registration_frame != h->last_registration) return OVGGT_ERR_INVALID_ARG;
+  }
   CK(cudaStreamSynchronize(h->last_stream));
   const int b = S.cur;
   const size_t row = (size_t)h->C * h->elem;
@@ -817,10 +840,35 @@ extern "C" int ovggt_cache_import(ovggt_cache* h, int32_t layer, const int64_t* 
   S.n_prot_hist = n_hist;
   S.pending_frame = next_frame_id - 1;
   S.frames_seen = n > 0 ? 1 : 0;
-  h->anchors.assign(anchor_frames.begin(), anchor_frames.end());
-  h->first_frame = n > 0 ? token_ids[0] / M : -1;
-  h->last_registration = n > 0 ? last_registration_frame : -1;
-  h->decided_frame = -1;
+  if (n > 0 && fresh) {
+    h->anchors.assign(anchor_frames.begin(), anchor_frames.end());
+    h->first_frame = token_ids[0] / M;
+    h->last_registration = last_registration_frame;
+    h->decided_frame = -1;
+  }
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_cache_reset(ovggt_cache* h) {
+  if (!h) return OVGGT_ERR_INVALID_ARG;
+  CK(cudaStreamSynchronize(h->last_stream));
+  if (h->side) CK(cudaStreamSynchronize(h->side));
+  for (LayerState& S : h->layers) {
+    S.n = 0;
+    S.cur = 0;
+    S.pending = false;
+    S.frames_seen = S.evicted_total = 0;
+    S.pending_frame = -1;
+    S.n_prot_init = S.n_prot_hist = 0;
+    S.last_N = S.last_keep = 0;
+    S.colsum_nparts = 0;
+    S.scores_frame = -1;
+  }
+  h->anchors.clear();
+  h->first_frame = h->last_registration = h->decided_frame = -1;
+  h->decided_register = false;
+  h->decided_demote = -1;
+  CK(cudaMemset(h->status, 0, 64));
   return OVGGT_OK;
 }
 

@@ -72,6 +72,13 @@ def test_create_reports_config_errors_without_a_gpu(lib):
         assert lib.ovggt_workspace_bytes(C.byref(cfg)) == 0
         assert lib.ovggt_cache_create(C.byref(cfg), C.byref(h)) == code
         assert not h.value
+    # a budget whose B + M candidates do not fit the selection cluster's shared memory is refused at create,
+    # not at the first step
+    huge = _cfg(n_heads=16, grid_h=37, grid_w=37, budget=120000, anchor_tokens=64, dtype=1)
+    assert lib.ovggt_workspace_bytes(C.byref(huge)) == 0
+    assert lib.ovggt_cache_create(C.byref(huge), C.byref(h)) == -10 and not h.value
+    assert lib.ovggt_workspace_bytes(C.byref(_cfg(n_heads=16, grid_h=37, grid_w=37, budget=65536, anchor_tokens=64,
+                                                  dtype=1))) > 0
     ok = _cfg(budget=69 + 3 * 8)
     assert lib.ovggt_workspace_bytes(C.byref(ok)) > 0
     assert lib.ovggt_cache_create(C.byref(ok), C.byref(h)) == -1          # no workspace given
@@ -89,6 +96,7 @@ def test_null_handle_and_strerror(lib):
         assert getattr(lib, name)(None, 0, C.byref(io), None) == -1
     st = B.OvggtStats()
     assert lib.ovggt_cache_stats(None, 0, C.byref(st)) == -1
+    assert lib.ovggt_cache_reset(None) == -1
     seen = {lib.ovggt_strerror(c) for c in range(0, -11, -1)}
     assert len(seen) == 11 and b"unknown error" not in seen
     assert lib.ovggt_strerror(-99) == b"unknown error"

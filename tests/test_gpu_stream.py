@@ -140,6 +140,83 @@ def test_export_import_roundtrip_and_resume():
     a.destroy(); b.destroy()
 
 
+def test_two_layer_export_import_resume_and_anchor_state_rules():
+    """The anchor FIFO belongs to the handle.  Two layers are exported in the middle of a stream with active
+    anchors, imported into a fresh handle (the first import brings the handle-wide state, the second must agree
+    with it) and both handles continue bit-identically.  Imports that disagree, and an empty import, leave the
+    handle-wide state untouched."""
+    cfg = gen.config_tiny().replace(n_layers=2, n_frames=12, tau=0.9, min_anchor_interval=2, k_max=2)
+    a = B.OvggtCache.from_stream(cfg)
+    frames = [[DeviceFrame(cfg, gen.frame_inputs(cfg, t, layer=l), "cuda") for l in range(2)] for t in range(cfg.n_frames)]
+
+    def step(c, t):
+        return [c.layer_step(l, t, f.q, f.k, f.v, f.resid, f.conf, f.rho) for l, f in enumerate(frames[t])]
+
+    for t in range(7):
+        step(a, t)
+    ex = [a.export(l) for l in range(2)]
+    sa = a.stats(0)
+    assert sa["n_active_anchors"] == 2                      # the FIFO is in use when the state is moved
+    last_reg = sa["anchor_frames"][-1]
+    b = B.OvggtCache.from_stream(cfg)
+    b.import_(0, ex[0]["ids"], ex[0]["flags"], ex[0]["stored"], ex[0]["k"], ex[0]["v"], 7, last_reg)
+    # an empty import of the other layer must not wipe what layer 0 brought
+    b.import_(1, ex[1]["ids"][:0], ex[1]["flags"][:0], ex[1]["stored"][:0], ex[1]["k"][:0], ex[1]["v"][:0], 7, last_reg)
+    assert b.stats(0)["anchor_frames"] == sa["anchor_frames"]
+    # a layer whose HIST rows name other frames than the handle's FIFO is refused
+    bad_flags = ex[1]["flags"].copy()
+    bad_flags[bad_flags == B.FLAG_HIST] = B.FLAG_EVICTABLE
+    with pytest.raises(B.OvggtError) as e:
+        b.import_(1, ex[1]["ids"], bad_flags, ex[1]["stored"], ex[1]["k"], ex[1]["v"], 7, last_reg)
+    assert e.value.code == -1
+    with pytest.raises(B.OvggtError):
+        b.import_(1, ex[1]["ids"], ex[1]["flags"], ex[1]["stored"], ex[1]["k"], ex[1]["v"], 7, last_reg - 1)
+    b.import_(1, ex[1]["ids"], ex[1]["flags"], ex[1]["stored"], ex[1]["k"], ex[1]["v"], 7, last_reg)
+    for l in range(2):
+        sb = b.stats(l)
+        assert sb["anchor_frames"] == sa["anchor_frames"]
+        assert (sb["n_protected_init"], sb["n_protected_hist"]) == (a.stats(l)["n_protected_init"], a.stats(l)["n_protected_hist"])
+    for t in range(7, cfg.n_frames):
+        for oa, ob in zip(step(a, t), step(b, t)):
+            assert torch.equal(oa, ob)
+    for l in range(2):
+        ea, eb = a.export(l), b.export(l)
+        for key in ea:
+            assert np.array_equal(ea[key], eb[key]), (l, key)
+        assert a.stats(l)["anchor_frames"] == b.stats(l)["anchor_frames"]
+    # reset empties the handle, after which another stream can be imported
+    b.reset()
+    assert b.stats(0)["n_cached"] == 0 and b.stats(0)["anchor_frames"] == []
+    b.import_(0, ex[0]["ids"], ex[0]["flags"], ex[0]["stored"], ex[0]["k"], ex[0]["v"], 7, last_reg)
+    assert b.stats(0)["anchor_frames"] == sa["anchor_frames"]
+    a.destroy(); b.destroy()
+
+
+def test_layers_must_compress_frames_in_order_across_the_handle():
+    """Layer 0 runs one frame ahead; layer 1 then comes with the older frame.  Its compress is refused (the anchor
+    decision of that frame cannot be taken twice) and the anchor state is what layer 0 left."""
+    cfg = gen.config_tiny().replace(n_layers=2, tau=0.95, min_anchor_interval=1, k_max=2)
+    c = B.OvggtCache.from_stream(cfg)
+    f = [[DeviceFrame(cfg, gen.frame_inputs(cfg, t, layer=l), "cuda") for l in range(2)] for t in range(4)]
+    for t in range(2):
+        for l in range(2):
+            x = f[t][l]
+            c.layer_step(l, t, x.q, x.k, x.v, x.resid, x.conf, x.rho)
+    x = f[2][0]
+    c.layer_attend(0, 2, x.q, x.k, x.v)
+    y = f[2][1]
+    c.layer_attend(1, 2, y.q, y.k, y.v)
+    c.layer_compress(0, 2, x.resid, x.conf, x.rho)
+    x3 = f[3][0]
+    c.layer_step(0, 3, x3.q, x3.k, x3.v, x3.resid, x3.conf, x3.rho)      # layer 0 is now ahead of layer 1
+    before = c.stats(0)["anchor_frames"]
+    with pytest.raises(B.OvggtError) as e:
+        c.layer_compress(1, 2, y.resid, y.conf, y.rho)
+    assert e.value.code == -4
+    assert c.stats(0)["anchor_frames"] == before
+    c.destroy()
+
+
 def test_call_order_errors():
     cfg = gen.config_tiny()
     c = B.OvggtCache.from_stream(cfg)
