@@ -60,6 +60,14 @@ enum {
 enum { OVGGT_DTYPE_F32 = 0, OVGGT_DTYPE_BF16 = 1 };
 enum { OVGGT_SCORE_HYBRID = 0, OVGGT_SCORE_RESIDUAL_STORED = 1 };
 enum { OVGGT_FLAG_EVICTABLE = 0, OVGGT_FLAG_INIT = 1, OVGGT_FLAG_HIST = 2 };
+/* Where surviving K/V rows live after Eq. 8 (the paper fixes the survivor set, not a layout):
+ *  FILL_HOLES     one K/V buffer per layer; the rows admitted from the new frame are copied into the slots the
+ *                 evicted rows leave (at most M rows move per step); logical (token id) order is kept in per-row
+ *                 meta and restored by ovggt_cache_export.  Attention reads the buffer front to back: the order of
+ *                 cached rows does not change its result beyond fp32 summation order.
+ *  STABLE_GATHER  two K/V buffers per layer; every survivor is copied, in token order, into the other buffer
+ *                 (B rows move per step; rows lie in token order on the device). */
+enum { OVGGT_COMPACT_FILL_HOLES = 0, OVGGT_COMPACT_STABLE_GATHER = 1 };
 
 typedef struct ovggt_cache ovggt_cache; /* opaque host-side handle */
 
@@ -74,6 +82,7 @@ typedef struct {
   int32_t protect_first_frame;           /* 1: Global Initial Anchor (all M first-frame tokens kept for good) */
   int32_t score_mode;                    /* OVGGT_SCORE_HYBRID (Eq. 7) or OVGGT_SCORE_RESIDUAL_STORED */
   int32_t dtype;                         /* OVGGT_DTYPE_* of q, k, v, resid, out and of the cache */
+  int32_t compaction;                    /* OVGGT_COMPACT_* */
   void* workspace;                       /* device, >= ovggt_workspace_bytes(cfg), 1024-byte aligned; need not be zeroed */
   size_t workspace_bytes;
 } ovggt_config;
@@ -100,7 +109,8 @@ typedef struct {
   int64_t evicted_total;        /* rows dropped so far */
   int32_t last_n_candidates;    /* N = n + M of the last step */
   int32_t last_n_survivors;     /* min(N, B) */
-  uint64_t bytes_resident;      /* workspace bytes this layer's K/V buffers occupy: constant over the stream */
+  uint64_t bytes_resident;      /* workspace bytes this layer's K/V buffers occupy: constant over the stream
+                                   (2 (B + M) C elements with hole filling, twice that with the stable gather) */
   int32_t device_status;        /* 0, or the OVGGT_ERR_* a kernel raised */
 } ovggt_stats;
 
@@ -130,10 +140,12 @@ int ovggt_layer_attend(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* 
  * score_override. */
 int ovggt_layer_compress(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
 
-/* ovggt_layer_attend and ovggt_layer_compress of one (frame, layer): the whole hot path.  The compress half reads
- * the cache and the new rows but not the attention's output, so it is enqueued on a second stream that the handle
- * owns (a host object, created by ovggt_cache_create), forked from and joined back into `stream` with events, and
- * runs beside the attention.  For the caller the call is still asynchronous and ordered on `stream` alone. */
+/* ovggt_layer_attend and ovggt_layer_compress of one (frame, layer): the whole hot path.  Scoring and selection
+ * read the cache and the new rows but not the attention's output, so they are enqueued on a second stream that the
+ * handle owns (a host object, created by ovggt_cache_create), forked from and joined back into `stream` with
+ * events, and run beside the attention; so does the stable gather, which writes another buffer.  The hole-filling
+ * move writes the buffer the attention reads and follows the join on `stream`.  For the caller the call is still
+ * asynchronous and ordered on `stream` alone. */
 int ovggt_layer_step(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
 
 /* Turn the overlap of ovggt_layer_step off (0) or on (non-zero, the default): off, the two halves run one after the
@@ -165,7 +177,10 @@ int ovggt_cache_export(ovggt_cache* cache, int32_t layer, int64_t* token_ids, ui
  * no frame adopts them from the first non-empty layer imported (FIFO = the frames of its HIST rows, oldest first;
  * first frame = its first row's frame; last_registration_frame as given); every later non-empty import must agree
  * with them (OVGGT_ERR_INVALID_ARG otherwise, nothing changed); an empty import never touches them.  To load a
- * different stream into a used handle, call ovggt_cache_reset first.  Synchronises. */
+ * different stream into a used handle, call ovggt_cache_reset first.  The imported rows lie in token order on the
+ * device.  With hole filling the exporting handle held the same rows in slot order, so the two handles add the
+ * attention's terms in different orders from then on: their outputs agree to fp32 rounding, not bit for bit (with the
+ * stable gather they are bit-identical).  Synchronises. */
 int ovggt_cache_import(ovggt_cache* cache, int32_t layer, const int64_t* token_ids, const uint8_t* flags,
                        const float* scores, const void* k, const void* v, int32_t n,
                        int64_t next_frame_id, int64_t last_registration_frame);

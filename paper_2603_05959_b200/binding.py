@@ -19,6 +19,7 @@ MAX_ANCHORS = 16
 DTYPE_F32, DTYPE_BF16 = 0, 1
 SCORE_HYBRID, SCORE_RESIDUAL_STORED = 0, 1
 FLAG_EVICTABLE, FLAG_INIT, FLAG_HIST = 0, 1, 2
+COMPACT_FILL_HOLES, COMPACT_STABLE_GATHER = 0, 1
 PROF_CLASSES = ["append", "attention", "row_norms", "diversity", "select", "compact"]
 
 EXPORTED = [
@@ -40,6 +41,7 @@ class OvggtConfig(C.Structure):
         ("anchor_tokens", C.c_int32), ("k_max", C.c_int32), ("min_anchor_interval", C.c_int32),
         ("tau", C.c_float), ("alpha", C.c_float), ("beta", C.c_float),
         ("protect_first_frame", C.c_int32), ("score_mode", C.c_int32), ("dtype", C.c_int32),
+        ("compaction", C.c_int32),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
     ]
 
@@ -150,13 +152,14 @@ class OvggtCache:
     def __init__(self, *, n_layers=1, n_heads=16, head_dim=64, n_special=5, grid_h=37, grid_w=37,
                  budget=16384, anchor_tokens=64, k_max=3, min_anchor_interval=100, tau=0.2, alpha=0.5,
                  beta=0.5, protect_first_frame=1, score_mode=SCORE_HYBRID, dtype=DTYPE_BF16,
-                 device: Optional[torch.device] = None):
+                 compaction=COMPACT_FILL_HOLES, device: Optional[torch.device] = None):
         budgets = [budget] * n_layers if isinstance(budget, int) else list(budget)
         assert len(budgets) == n_layers
         self._budgets = (C.c_int32 * n_layers)(*budgets)
         self.cfg = OvggtConfig(n_layers, n_heads, head_dim, n_special, grid_h, grid_w, self._budgets,
                                anchor_tokens, k_max, min_anchor_interval, tau, alpha, beta,
-                               protect_first_frame, score_mode, dtype, None, 0)
+                               protect_first_frame, score_mode, dtype, compaction, None, 0)
+        self.compaction = compaction
         self.M = n_special + grid_h * grid_w
         self.C = n_heads * head_dim
         self.n_patches = grid_h * grid_w

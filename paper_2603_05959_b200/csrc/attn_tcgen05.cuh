@@ -695,16 +695,37 @@ inline size_t attn_tcgen05_scratch_bytes(int M, int N, int H) {
 
 inline int attn_tcgen05_num_launches(int M, int N, int H) { return attn_choose_splits(M, N, H) > 1 ? 2 : 1; }
 
+// Tensor maps of a K/V buffer pair, kept by the caller between launches: a cache that lives in one buffer with a
+// row count that stops changing needs them encoded once, not once per step.
+struct AttnKvMaps {
+  CUtensorMap k, v;
+  const void *k_base = nullptr, *v_base = nullptr;
+  int rows = -1, C = 0;
+};
+
+inline int attn_kv_maps(AttnKvMaps* m, const void* k, const void* v, int N, int C) {
+  if (m->k_base == k && m->v_base == v && m->rows == N && m->C == C) return OVGGT_OK;
+  m->rows = -1;
+  int rc = make_rows_map(&m->k, k, N, C, kBN);
+  if (rc) return rc;
+  rc = make_rows_map(&m->v, v, N, C, kBN);
+  if (rc) return rc;
+  m->k_base = k; m->v_base = v; m->rows = N; m->C = C;
+  return OVGGT_OK;
+}
+
 inline int attn_tcgen05_launch(const void* q, const void* k, const void* v, int M, int N, int H, void* out,
-                               void* scratch, int* status, cudaStream_t st) {
+                               void* scratch, int* status, cudaStream_t st, AttnKvMaps* kv_maps = nullptr) {
   const int C = H * kHD;
-  CUtensorMap tq, tk, tv;
+  CUtensorMap tq;
+  AttnKvMaps local;
+  AttnKvMaps* maps = kv_maps ? kv_maps : &local;
   int rc = make_rows_map(&tq, q, M, C, kBM);
   if (rc) return rc;
-  rc = make_rows_map(&tk, k, N, C, kBN);
+  rc = attn_kv_maps(maps, k, v, N, C);
   if (rc) return rc;
-  rc = make_rows_map(&tv, v, N, C, kBN);
-  if (rc) return rc;
+  const CUtensorMap& tk = maps->k;
+  const CUtensorMap& tv = maps->v;
   AttnParams P;
   P.M = M; P.N = N; P.H = H;
   P.tiles_total = (N + kBN - 1) / kBN;

@@ -3,6 +3,8 @@
 // loads issued before its stores, so many independent 16-byte transactions are in flight per SM.
 #pragma once
 
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace ovggt {
@@ -114,12 +116,13 @@ __global__ void __launch_bounds__(256) k_compact_colsum(const uint4* __restrict_
     part[(size_t)blockIdx.x * C + c] = ((red[0][c] + red[1][c]) + red[2][c]) + red[3][c];
 }
 
-// Rows [n, n+M) of the cache := the frame's K and V; their meta: ids frame*M + j, evictable, score 0.
+// Rows [n, n+M) of the cache := the frame's K and V; their meta: ids frame*M + j, evictable, score 0 and, in the
+// hole-filling layout (slot != nullptr), the physical slot n + j.
 __global__ void __launch_bounds__(256) k_append(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
                                                 int M, int nvec, int n, long long frame_id,
                                                 uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
                                                 long long* __restrict__ ids, uint8_t* __restrict__ flags,
-                                                float* __restrict__ stored) {
+                                                float* __restrict__ stored, int* __restrict__ slot) {
   const int lane = threadIdx.x & 31;
   const int gtid = blockIdx.x * blockDim.x + threadIdx.x;
   const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
@@ -132,7 +135,107 @@ __global__ void __launch_bounds__(256) k_append(const uint4* __restrict__ k_new,
     ids[n + j] = frame_id * (long long)M + j;
     flags[n + j] = OVGGT_FLAG_EVICTABLE;
     stored[n + j] = 0.0f;
+    if (slot) slot[n + j] = n + j;
   }
+}
+
+// ---- hole-filling compaction (Eq. 8 fixes the survivor set, not where the rows live)
+//
+// The selection kernel leaves n_moves pairs: the K/V row in slot move_src[i] (a survivor above slot B) goes to
+// slot move_dst[i] (a slot below B whose row was evicted), and the survivor's meta entry move_j[i] learns its new
+// slot.  Nothing else moves, so a step at steady state copies at most M rows instead of B.
+// With `delta` the kernel also leaves what the move does to the column sums of the keys in slots [0, B):
+//   delta[c] = sum_i (K[move_src[i], c] - K[move_dst[i], c])     (keys admitted minus keys evicted)
+// as kFillSlices partial rows, one per 8-CTA cluster: a warp folds its moves in order, the CTA folds its warps in
+// order, the cluster folds its CTAs in rank order through distributed shared memory.  The next step's diversity
+// kernel adds the slices, in slice order, to the sums it used this step, so no pass over all keys is needed and the
+// result does not depend on timing.  Requires nvec <= kCompactSumMaxVec when delta is asked for.
+constexpr int kFillSlices = 16;
+constexpr int kFillClusterCtas = 8;
+constexpr int kFillThreads = 256;
+
+template <int DT>
+__global__ void __launch_bounds__(kFillThreads) k_fill_holes(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
+                                                             const int* __restrict__ move_src,
+                                                             const int* __restrict__ move_dst,
+                                                             const int* __restrict__ move_j,
+                                                             const int* __restrict__ n_moves_ptr, int max_moves,
+                                                             int nvec, int* __restrict__ slot_meta,
+                                                             float* __restrict__ delta /* [kFillSlices, C] or null */) {
+  constexpr int VEC = VecOf<DT>::n;
+  __shared__ __align__(16) float red[4][kCompactSumMaxVec * VEC];
+  __shared__ __align__(16) float cta_part[kCompactSumMaxVec * VEC];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
+  const int n_moves = min(*n_moves_ptr, max_moves);
+  const bool sum = delta != nullptr;
+  float acc[4][VEC];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[i][e] = 0.0f;
+  for (int m = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5); m < n_moves; m += warps_total) {
+    const int src = move_src[m], dst = move_dst[m];
+    for (int v0 = lane; v0 < nvec; v0 += 128) {
+      uint4 uk[4], uv[4], uo[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (v0 + 32 * i < nvec) {
+          uk[i] = ld_nc(k_cache + (size_t)src * nvec + v0 + 32 * i);
+          uv[i] = ld_nc(v_cache + (size_t)src * nvec + v0 + 32 * i);
+          if (sum) uo[i] = ld_nc(k_cache + (size_t)dst * nvec + v0 + 32 * i);
+        }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (v0 + 32 * i < nvec) {
+          k_cache[(size_t)dst * nvec + v0 + 32 * i] = uk[i];
+          v_cache[(size_t)dst * nvec + v0 + 32 * i] = uv[i];
+          if (sum) {
+            float a[VEC], b[VEC];
+            unpack<DT>(uk[i], a);
+            unpack<DT>(uo[i], b);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[i][e] += a[e] - b[e];
+          }
+        }
+    }
+    if (lane == 0) slot_meta[move_j[m]] = dst;
+  }
+  if (!sum) return;
+  // CTA fold: warps 4..7 park, 0..3 add their own, then the four are added in order (as in k_compact_colsum)
+  auto park = [&](int slot, bool add) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (lane + 32 * i < nvec)
+#pragma unroll
+        for (int e = 0; e < VEC; e += 4) {
+          float4* p = reinterpret_cast<float4*>(&red[slot][(lane + 32 * i) * VEC + e]);
+          float4 t = make_float4(acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]);
+          if (add) {
+            const float4 o = *p;
+            t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
+          }
+          *p = t;
+        }
+  };
+  if (warp >= 4) park(warp - 4, false);
+  __syncthreads();
+  if (warp < 4) park(warp, true);
+  __syncthreads();
+  const int C = nvec * VEC;
+  for (int c = threadIdx.x; c < C; c += blockDim.x) cta_part[c] = ((red[0][c] + red[1][c]) + red[2][c]) + red[3][c];
+  // cluster fold through distributed shared memory: CTA r of the cluster owns every 8th group of 32 columns
+  cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
+  cluster.sync();
+  const int ncta = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+  const int cid = (int)blockIdx.x / ncta;
+  for (int c = rank * 32 + (threadIdx.x & 31) + (threadIdx.x >> 5) * 32 * ncta; c < C;
+       c += 32 * ncta * (blockDim.x >> 5)) {
+    float t = 0.0f;
+    for (int q = 0; q < ncta; ++q) t += cluster.map_shared_rank(cta_part, q)[c];
+    delta[(size_t)cid * C + c] = t;
+  }
+  cluster.sync();   // no CTA may exit while others still read its shared memory
 }
 
 }  // namespace ovggt

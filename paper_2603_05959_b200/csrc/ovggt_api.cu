@@ -99,9 +99,11 @@ int launch_diversity(const void* K, int rows, int C, int dtype, float* part, flo
   const int grid = std::min((rows + 7) / 8, 148 * 8);
   const size_t smem = (size_t)C * 4;
   if (dtype == kBF16)
-    k_diversity<kBF16><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d, grid, nullptr, 0, nullptr);
+    k_diversity<kBF16><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, nullptr, d, grid, nullptr, 0,
+                                                nullptr);
   else
-    k_diversity<kF32><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d, grid, nullptr, 0, nullptr);
+    k_diversity<kF32><<<grid, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, nullptr, d, grid, nullptr, 0,
+                                               nullptr);
   LAUNCHED();
   return OVGGT_OK;
 }
@@ -125,10 +127,10 @@ int launch_diversity_from_parts(const void* K, int rows, int C, int dtype, const
   const size_t smem = (size_t)C * 4;
   const int norm_ctas = resid ? (resid_rows + 7) / 8 : 0;
   if (dtype == kBF16)
-    k_diversity<kBF16><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d, grid,
+    k_diversity<kBF16><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, nullptr, d, grid,
                                                             (const uint4*)resid, resid_rows, s_raw);
   else
-    k_diversity<kF32><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, d, grid,
+    k_diversity<kF32><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, 1, nullptr, d, grid,
                                                            (const uint4*)resid, resid_rows, s_raw);
   LAUNCHED();
   return OVGGT_OK;
@@ -162,10 +164,71 @@ int launch_compact(const void* ks, const void* vs, const int* surv, int n_keep, 
   return OVGGT_OK;
 }
 
+// Diversity against sums given as n_slices rows (see k_diversity); the frame's residual norms ride in the same
+// launch when resid is given; the folded sums go to ksum_out when it is given.
+int launch_diversity_sliced(const void* K, int rows, int C, int dtype, const float* ksum, int n_slices, float* ksum_out,
+                            float* d, const void* resid, int resid_rows, float* s_raw, cudaStream_t st) {
+  if (rows <= 0) return OVGGT_OK;
+  const int nvec = C * elem_bytes(dtype) / 16;
+  const int grid = std::min((rows + 63) / 64, 148 * 8);
+  const size_t smem = (size_t)C * 4;
+  const int norm_ctas = resid ? (resid_rows + 7) / 8 : 0;
+  if (dtype == kBF16)
+    k_diversity<kBF16><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, n_slices, ksum_out, d,
+                                                            grid, (const uint4*)resid, resid_rows, s_raw);
+  else
+    k_diversity<kF32><<<grid + norm_ctas, 256, smem, st>>>((const uint4*)K, rows, nvec, ksum, n_slices, ksum_out, d,
+                                                           grid, (const uint4*)resid, resid_rows, s_raw);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
+// Column sums of K [rows, C] into ksum [C] (two kernels; part: [colsum_parts(rows), C] floats of scratch).
+int launch_colsum(const void* K, int rows, int C, int dtype, float* part, float* ksum, cudaStream_t st) {
+  const int nvec = C * elem_bytes(dtype) / 16;
+  const int parts = colsum_parts(rows);
+  const int rpc = (rows + parts - 1) / parts;
+  const int threads = std::min(256, (nvec + 31) / 32 * 32);
+  if (dtype == kBF16) k_colsum_partial<kBF16><<<parts, threads, 0, st>>>((const uint4*)K, rows, nvec, rpc, part);
+  else                k_colsum_partial<kF32><<<parts, threads, 0, st>>>((const uint4*)K, rows, nvec, rpc, part);
+  LAUNCHED();
+  k_colsum_final<<<(C + 31) / 32, 1024, 0, st>>>(part, parts, C, ksum);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
+// The hole-filling move (and, with delta, what it does to the key column sums).
+int launch_fill_holes(void* kc, void* vc, const int* msrc, const int* mdst, const int* mj, const int* n_moves, int max_moves,
+                      int C, int dtype, int* slot_meta, float* delta, cudaStream_t st) {
+  const int nvec = C * elem_bytes(dtype) / 16;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kFillSlices * kFillClusterCtas);
+  cfg.blockDim = dim3(kFillThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = kFillClusterCtas;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaError_t e;
+  if (dtype == kBF16)
+    e = cudaLaunchKernelEx(&cfg, k_fill_holes<kBF16>, (uint4*)kc, (uint4*)vc, msrc, mdst, mj, n_moves, max_moves, nvec,
+                           slot_meta, delta);
+  else
+    e = cudaLaunchKernelEx(&cfg, k_fill_holes<kF32>, (uint4*)kc, (uint4*)vc, msrc, mdst, mj, n_moves, max_moves, nvec,
+                           slot_meta, delta);
+  if (e != cudaSuccess) return cuda_fail(e);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
 int launch_attention(const void* q, const void* k, const void* v, int M, int N, int H, int dtype, void* out,
-                     void* scratch, int* status, cudaStream_t st) {
+                     void* scratch, int* status, cudaStream_t st, AttnKvMaps* maps = nullptr) {
   if (dtype == kBF16) {
-    int rc = attn_tcgen05_launch(q, k, v, M, N, H, out, scratch, status, st);
+    int rc = attn_tcgen05_launch(q, k, v, M, N, H, out, scratch, status, st, maps);
     if (rc == OVGGT_OK) g_launches.fetch_add(attn_tcgen05_num_launches(M, N, H));
     if (rc == OVGGT_ERR_CUDA) g_last_cuda_error.store(attn_tcgen05_last_error());
     return rc;
@@ -180,10 +243,15 @@ int launch_attention(const void* q, const void* k, const void* v, int M, int N, 
 
 // ------------------------------------------------------------------ handle
 
+// Steps between two full recomputations of the key column sums in the hole-filling layout: in between, the sums
+// follow the cache by "+ admitted - evicted" corrections, whose fp32 rounding (about 1e-7 relative per step) adds up.
+constexpr int kColsumRefreshEvery = 64;
+
 struct LayerState {
   int budget = 0;
   int n = 0;            // rows held between steps
-  int cur = 0;          // which of the two buffers holds them
+  int cur = 0;          // which of the two meta buffers (ids, flags, stored scores, slots) describes them
+  int kv = 0;           // which K/V buffer holds them (always 0 in the hole-filling layout)
   bool pending = false; // a frame was appended and not yet compressed
   int64_t frames_seen = 0, evicted_total = 0, pending_frame = -1;
   int n_prot_init = 0, n_prot_hist = 0;
@@ -194,11 +262,19 @@ struct LayerState {
   long long* ids[2];
   uint8_t* flags[2];
   float* stored[2];
+  int* slot[2] = {nullptr, nullptr};   // hole-filling layout: physical K/V slot of each logical row
   float *s_raw, *d, *r;
   int* surv;
   int* n_keep_dev;
-  float* colsum_part = nullptr;   // [148 * 8, C]: per-CTA column sums of the keys the last compaction wrote
+  float* colsum_part = nullptr;   // stable layout: [148 * 8, C] per-CTA column sums of the keys the last compaction wrote
   int colsum_nparts = 0;          // 0: not available (the next step sums the keys itself)
+  // hole-filling layout
+  int *move_src = nullptr, *move_dst = nullptr, *move_j = nullptr, *n_moves_dev = nullptr;
+  float* ksum[2] = {nullptr, nullptr};   // [1 + kFillSlices, C]: the key column sums a step uses, then the move's corrections
+  int kcur = 0;                   // which of the two the next diversity launch reads
+  bool ksum_valid = false;        // ksum[kcur] describes the cached keys (else: recompute)
+  int since_refresh = 0;
+  AttnKvMaps maps[2];             // tensor maps of the K/V buffers, re-encoded only when the row count changes
   int64_t scores_frame = -1;      // frame whose s_raw and d were already enqueued on the side stream
   size_t kv_bytes = 0;
 };
@@ -283,6 +359,7 @@ bool config_ok(const ovggt_config* c, int* err) {
   if (c->k_max < 0 || c->k_max > OVGGT_MAX_ANCHORS || c->min_anchor_interval < 0) return false;
   if (c->dtype != kF32 && c->dtype != kBF16) return false;
   if (c->score_mode != OVGGT_SCORE_HYBRID && c->score_mode != OVGGT_SCORE_RESIDUAL_STORED) return false;
+  if (c->compaction != OVGGT_COMPACT_FILL_HOLES && c->compaction != OVGGT_COMPACT_STABLE_GATHER) return false;
   if (!(c->alpha >= 0.0f && c->alpha <= 1.0f) || !(c->beta >= 0.0f && c->beta <= 1.0f)) return false;
   const int64_t M = c->n_special + (int64_t)c->grid_h * c->grid_w;
   const int64_t pmax = (c->protect_first_frame ? M : 0) + (int64_t)c->k_max * c->anchor_tokens;
@@ -314,10 +391,12 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
   for (int l = 0; l < c->n_layers; ++l) {
     const size_t R = (size_t)c->budget[l] + M;
     max_rows = std::max(max_rows, (int)R);
-    size_t off[20];
+    const bool fill = c->compaction == OVGGT_COMPACT_FILL_HOLES;
+    const int nkv = fill ? 1 : 2;       // the stable gather writes the other buffer of a pair; hole filling moves in place
+    size_t off[32];
     int i = 0;
-    for (int b = 0; b < 2; ++b) off[i++] = L.take(R * C * eb);
-    for (int b = 0; b < 2; ++b) off[i++] = L.take(R * C * eb);
+    for (int b = 0; b < nkv; ++b) off[i++] = L.take(R * C * eb);
+    for (int b = 0; b < nkv; ++b) off[i++] = L.take(R * C * eb);
     for (int b = 0; b < 2; ++b) off[i++] = L.take(R * 8);
     for (int b = 0; b < 2; ++b) off[i++] = L.take(R);
     for (int b = 0; b < 2; ++b) off[i++] = L.take(R * 4);
@@ -325,13 +404,20 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
     off[i++] = L.take(R * 4);           // d
     off[i++] = L.take(R * 4);           // r
     off[i++] = L.take(R * 4);           // survivors
-    off[i++] = L.take(64);              // n_keep
-    off[i++] = L.take((size_t)148 * 8 * C * 4);   // column-sum partials of the compaction
+    off[i++] = L.take(64);              // n_keep, n_moves
+    if (fill) {
+      for (int b = 0; b < 2; ++b) off[i++] = L.take(R * 4);                                  // slots
+      for (int b = 0; b < 3; ++b) off[i++] = L.take((size_t)M * 4);                          // move lists
+      for (int b = 0; b < 2; ++b) off[i++] = L.take((size_t)(1 + kFillSlices) * C * 4);      // column sums + corrections
+    } else {
+      off[i++] = L.take((size_t)148 * 8 * C * 4);   // column-sum partials of the compaction
+    }
     if (h) {
       LayerState& S = h->layers[l];
       i = 0;
-      for (int b = 0; b < 2; ++b) S.kbuf[b] = base + off[i++];
-      for (int b = 0; b < 2; ++b) S.vbuf[b] = base + off[i++];
+      S.kbuf[1] = S.vbuf[1] = nullptr;
+      for (int b = 0; b < nkv; ++b) S.kbuf[b] = base + off[i++];
+      for (int b = 0; b < nkv; ++b) S.vbuf[b] = base + off[i++];
       for (int b = 0; b < 2; ++b) S.ids[b] = reinterpret_cast<long long*>(base + off[i++]);
       for (int b = 0; b < 2; ++b) S.flags[b] = reinterpret_cast<uint8_t*>(base + off[i++]);
       for (int b = 0; b < 2; ++b) S.stored[b] = reinterpret_cast<float*>(base + off[i++]);
@@ -340,9 +426,18 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
       S.r = reinterpret_cast<float*>(base + off[i++]);
       S.surv = reinterpret_cast<int*>(base + off[i++]);
       S.n_keep_dev = reinterpret_cast<int*>(base + off[i++]);
-      S.colsum_part = reinterpret_cast<float*>(base + off[i++]);
+      S.n_moves_dev = S.n_keep_dev + 4;
+      if (fill) {
+        for (int b = 0; b < 2; ++b) S.slot[b] = reinterpret_cast<int*>(base + off[i++]);
+        S.move_src = reinterpret_cast<int*>(base + off[i++]);
+        S.move_dst = reinterpret_cast<int*>(base + off[i++]);
+        S.move_j = reinterpret_cast<int*>(base + off[i++]);
+        for (int b = 0; b < 2; ++b) S.ksum[b] = reinterpret_cast<float*>(base + off[i++]);
+      } else {
+        S.colsum_part = reinterpret_cast<float*>(base + off[i++]);
+      }
       S.budget = c->budget[l];
-      S.kv_bytes = 4 * R * C * eb;
+      S.kv_bytes = 2 * (size_t)nkv * R * C * eb;
     }
   }
   const size_t o_part = L.take((size_t)kMaxColsumParts * C * 4);
@@ -480,35 +575,46 @@ extern "C" int ovggt_cache_destroy(ovggt_cache* h) {
 }
 
 namespace {
-// Eq. 2: validation of the attend half and the append itself.
-int enqueue_append(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st) {
+inline bool fill_layout(const ovggt_cache* h) { return h->cfg.compaction == OVGGT_COMPACT_FILL_HOLES; }
+
+// Argument and order checks of the attend half.
+int validate_attend(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io) {
   int rc = check_layer(h, layer);
   if (rc) return rc;
   if (!io || !io->q || !io->k || !io->v || !io->out) return OVGGT_ERR_INVALID_ARG;
   if (!aligned16(io->q) || !aligned16(io->k) || !aligned16(io->v) || !aligned16(io->out)) return OVGGT_ERR_MISALIGNED;
-  LayerState& S = h->layers[layer];
+  const LayerState& S = h->layers[layer];
   if (S.pending) return OVGGT_ERR_FRAME_ORDER;
   if (S.frames_seen > 0 && io->frame_id <= S.pending_frame) return OVGGT_ERR_FRAME_ORDER;
   if (io->frame_id < 0 || (h->first_frame >= 0 && io->frame_id < h->first_frame)) return OVGGT_ERR_FRAME_ORDER;
+  return OVGGT_OK;
+}
+
+// Eq. 2: the append itself.
+int enqueue_append(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st) {
+  int rc = validate_attend(h, layer, io);
+  if (rc) return rc;
+  LayerState& S = h->layers[layer];
   h->last_stream = st;
-  const int M = h->M, C = h->C, nvec = C * h->elem / 16, b = S.cur;
+  const int M = h->M, C = h->C, nvec = C * h->elem / 16, b = S.cur, kb = S.kv;
   const int grid = std::min((2 * M + 7) / 8, 148 * 8);
   ProfScope ps(h, OVGGT_PROF_APPEND, st);
   k_append<<<grid, 256, 0, st>>>((const uint4*)io->k, (const uint4*)io->v, M, nvec, S.n, (long long)io->frame_id,
-                                 (uint4*)S.kbuf[b], (uint4*)S.vbuf[b], S.ids[b], S.flags[b], S.stored[b]);
+                                 (uint4*)S.kbuf[kb], (uint4*)S.vbuf[kb], S.ids[b], S.flags[b], S.stored[b], S.slot[b]);
   LAUNCHED();
   return OVGGT_OK;
 }
 
-// The attention over all n + M rows, and the bookkeeping that closes the attend half.
+// The attention over all n + M rows, and the bookkeeping that closes the attend half.  Attention does not care in
+// which order the cached rows lie, so it reads the K/V buffer front to back in either layout.
 int enqueue_attention(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st) {
   LayerState& S = h->layers[layer];
-  const int b = S.cur;
+  const int kb = S.kv;
   int rc;
   {
     ProfScope ps(h, OVGGT_PROF_ATTENTION, st);
-    rc = launch_attention(io->q, S.kbuf[b], S.vbuf[b], h->M, S.n + h->M, h->cfg.n_heads, h->cfg.dtype, io->out,
-                          h->attn_scratch, h->status, st);
+    rc = launch_attention(io->q, S.kbuf[kb], S.vbuf[kb], h->M, S.n + h->M, h->cfg.n_heads, h->cfg.dtype, io->out,
+                          h->attn_scratch, h->status, st, &S.maps[kb]);
   }
   if (rc) return rc;
   if (h->first_frame < 0) {
@@ -519,28 +625,64 @@ int enqueue_attention(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, c
   S.pending_frame = io->frame_id;
   return OVGGT_OK;
 }
-}  // namespace
 
-extern "C" int ovggt_layer_attend(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  int rc = enqueue_append(h, layer, io, st);
+// Eq. 5 and the diversity score of Sec. 3.2 for the frame io describes: everything the selection needs that does not
+// depend on the anchor decision.  Reads the cached keys [0, n) and the frame's residual, so it may run before the
+// frame's K/V are appended.
+int enqueue_scores(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io, cudaStream_t st) {
+  const ovggt_config& c = h->cfg;
+  const int M = h->M, C = h->C, n = S.n, kb = S.kv;
+  const bool hybrid = c.score_mode == OVGGT_SCORE_HYBRID && n > 0;
+  int rc = OVGGT_OK;
+  if (!hybrid) {
+    ProfScope ps(h, OVGGT_PROF_ROW_NORMS, st);
+    return launch_row_norms(io->resid, M, C, c.dtype, S.s_raw, st);
+  }
+  if (fill_layout(h)) {
+    // Column sums of the cached keys: continued from the last step's sums and the corrections its move left, or
+    // summed afresh (first steps, after an import, every kColsumRefreshEvery-th step); the residual norms ride in
+    // the diversity launch either way.
+    ProfScope ps(h, OVGGT_PROF_DIVERSITY, st);
+    const bool fresh = !S.ksum_valid || S.since_refresh >= kColsumRefreshEvery;
+    if (fresh) {
+      rc = launch_colsum(S.kbuf[kb], n, C, c.dtype, h->colsum_part, S.ksum[S.kcur], st);
+      if (rc) return rc;
+      S.since_refresh = 0;
+    } else {
+      S.since_refresh += 1;
+    }
+    return launch_diversity_sliced(S.kbuf[kb], n, C, c.dtype, S.ksum[S.kcur], fresh ? 1 : 1 + kFillSlices,
+                                   S.ksum[S.kcur ^ 1], S.d, io->resid, M, S.s_raw, st);
+  }
+  if (S.colsum_nparts > 0) {   // stable layout, sums left by the last compaction
+    ProfScope ps(h, OVGGT_PROF_DIVERSITY, st);
+    return launch_diversity_from_parts(S.kbuf[kb], n, C, c.dtype, S.colsum_part, S.colsum_nparts, h->ksum, S.d,
+                                       io->resid, M, S.s_raw, st);
+  }
+  {
+    ProfScope ps(h, OVGGT_PROF_ROW_NORMS, st);
+    rc = launch_row_norms(io->resid, M, C, c.dtype, S.s_raw, st);
+  }
   if (rc) return rc;
-  return enqueue_attention(h, layer, io, st);
+  ProfScope ps(h, OVGGT_PROF_DIVERSITY, st);
+  return launch_diversity(S.kbuf[kb], n, C, c.dtype, h->colsum_part, h->ksum, S.d, st);
 }
 
-extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
+// The compress half.  Scores and selection go to st_sel.  What moves K/V rows goes to st_move: the stable gather
+// writes another buffer and may run beside an attention that still reads this one (st_move = st_sel); the
+// hole-filling move writes the buffer the attention reads, so it follows both (st_move = the attention's stream,
+// which first waits for st_sel).
+int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st_sel, cudaStream_t st_move) {
   int rc = check_layer(h, layer);
   if (rc) return rc;
   if (!io || !io->resid) return OVGGT_ERR_INVALID_ARG;
   if (!aligned16(io->resid)) return OVGGT_ERR_MISALIGNED;
   LayerState& S = h->layers[layer];
   if (!S.pending || io->frame_id != S.pending_frame) return OVGGT_ERR_FRAME_ORDER;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  h->last_stream = st;
   const ovggt_config& c = h->cfg;
-  const int M = h->M, C = h->C, n = S.n, N = n + M, B = S.budget, b = S.cur;
+  const int M = h->M, C = h->C, n = S.n, N = n + M, B = S.budget, b = S.cur, kb = S.kv;
   const int64_t t = io->frame_id;
-
+  const bool fill = fill_layout(h);
   const int ncta = select_cluster_ctas(N);
   const size_t smem = compress_smem_bytes((N + ncta - 1) / ncta, h->Np, M);
   if (smem > kSmemLimit) return OVGGT_ERR_UNSUPPORTED;   // (create already refuses such budgets)
@@ -566,25 +708,12 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
     }
   }
   const bool first = (t == h->first_frame);
+  h->last_stream = st_move;
 
-  // With column sums left by the last compaction, the residual norms ride in the diversity launch.
-  const bool fused_scores = c.score_mode == OVGGT_SCORE_HYBRID && n > 0 && S.colsum_nparts > 0;
-  const bool prelaunched = S.scores_frame == t;    // ovggt_layer_step already enqueued them on the side stream
+  const bool prelaunched = S.scores_frame == t;    // ovggt_layer_step already enqueued them on st_sel
   S.scores_frame = -1;
-  if (prelaunched) {
-    // (enqueued earlier on this same stream by ovggt_layer_step)
-  } else if (!fused_scores) {
-    ProfScope ps(h, OVGGT_PROF_ROW_NORMS, st);
-    rc = launch_row_norms(io->resid, M, C, c.dtype, S.s_raw, st);
-  }
-  if (rc) return rc;
-  if (c.score_mode == OVGGT_SCORE_HYBRID && n > 0 && !prelaunched) {
-    ProfScope ps(h, OVGGT_PROF_DIVERSITY, st);
-    if (fused_scores)
-      rc = launch_diversity_from_parts(S.kbuf[b], n, C, c.dtype, S.colsum_part, S.colsum_nparts, h->ksum, S.d,
-                                       io->resid, M, S.s_raw, st);
-    else
-      rc = launch_diversity(S.kbuf[b], n, C, c.dtype, h->colsum_part, h->ksum, S.d, st);
+  if (!prelaunched) {
+    rc = enqueue_scores(h, S, io, st_sel);
     if (rc) return rc;
   }
   CompressParams P;
@@ -602,24 +731,48 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
   P.ids_dst = S.ids[b ^ 1]; P.flags_dst = S.flags[b ^ 1]; P.stored_dst = S.stored[b ^ 1];
   P.r_out = S.r; P.survivors = S.surv;
   P.status = h->status; P.n_keep_out = S.n_keep_dev;
+  P.fill = fill ? 1 : 0;
+  P.slot_src = S.slot[b]; P.slot_dst = S.slot[b ^ 1];
+  P.move_src = S.move_src; P.move_dst = S.move_dst; P.move_j = S.move_j; P.n_moves_out = S.n_moves_dev;
   CK(cudaFuncSetAttribute(k_compress_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit));
   {
-    ProfScope ps(h, OVGGT_PROF_SELECT, st);
-    CK(launch_cluster(k_compress_select, dim3(ncta), ncta, smem, st, P));
+    ProfScope ps(h, OVGGT_PROF_SELECT, st_sel);
+    CK(launch_cluster(k_compress_select, dim3(ncta), ncta, smem, st_sel, P));
     LAUNCHED();
   }
   const int n_keep = std::min(N, B);
-  {
-    ProfScope ps(h, OVGGT_PROF_COMPACT, st);
-    const bool fuse = c.score_mode == OVGGT_SCORE_HYBRID && C * h->elem / 16 <= kCompactSumMaxVec;
+  const bool sums_fit = C * h->elem / 16 <= kCompactSumMaxVec;
+  if (fill) {
+    S.ksum_valid = false;
+    if (N > B) {   // some rows leave: survivors above slot B move into the slots that open below it
+      if (st_move != st_sel) {
+        CK(cudaEventRecord(h->ev_join, st_sel));
+        CK(cudaStreamWaitEvent(st_move, h->ev_join, 0));
+      }
+      // The corrections continue the sums this step's diversity launch used and wrote to ksum[kcur ^ 1]; they
+      // describe the next cache only if every slot below B held a cached row (n == B: steady state).
+      const bool delta = c.score_mode == OVGGT_SCORE_HYBRID && sums_fit && n == B;
+      ProfScope ps(h, OVGGT_PROF_COMPACT, st_move);
+      rc = launch_fill_holes(S.kbuf[kb], S.vbuf[kb], S.move_src, S.move_dst, S.move_j, S.n_moves_dev, M, C, c.dtype,
+                             S.slot[b ^ 1], delta ? S.ksum[S.kcur ^ 1] + C : nullptr, st_move);
+      if (rc) return rc;
+      if (delta) {
+        S.kcur ^= 1;
+        S.ksum_valid = true;
+      }
+    }
+  } else {
+    ProfScope ps(h, OVGGT_PROF_COMPACT, st_move);
+    const bool fuse = c.score_mode == OVGGT_SCORE_HYBRID && sums_fit;
     S.colsum_nparts = 0;
     if (fuse)
-      rc = launch_compact_colsum(S.kbuf[b], S.vbuf[b], S.surv, n_keep, C, c.dtype, S.kbuf[b ^ 1], S.vbuf[b ^ 1],
-                                 S.colsum_part, &S.colsum_nparts, st);
+      rc = launch_compact_colsum(S.kbuf[kb], S.vbuf[kb], S.surv, n_keep, C, c.dtype, S.kbuf[kb ^ 1], S.vbuf[kb ^ 1],
+                                 S.colsum_part, &S.colsum_nparts, st_move);
     else
-      rc = launch_compact(S.kbuf[b], S.vbuf[b], S.surv, n_keep, C, c.dtype, S.kbuf[b ^ 1], S.vbuf[b ^ 1], st);
+      rc = launch_compact(S.kbuf[kb], S.vbuf[kb], S.surv, n_keep, C, c.dtype, S.kbuf[kb ^ 1], S.vbuf[kb ^ 1], st_move);
+    if (rc) return rc;
+    S.kv = kb ^ 1;
   }
-  if (rc) return rc;
 
   // bookkeeping that follows deterministically from the sizes
   if (first && c.protect_first_frame) S.n_prot_init = M;
@@ -634,6 +787,19 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
   S.frames_seen += 1;
   return OVGGT_OK;
 }
+}  // namespace
+
+extern "C" int ovggt_layer_attend(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = enqueue_append(h, layer, io, st);
+  if (rc) return rc;
+  return enqueue_attention(h, layer, io, st);
+}
+
+extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return compress_impl(h, layer, io, st, st);
+}
 
 extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
   int rc = check_layer(h, layer);
@@ -646,30 +812,27 @@ extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame
     if (rc) return rc;
     return ovggt_layer_compress(h, layer, io, stream);
   }
-  // Scoring, selection and compaction (Eq. 5-8) read the cache and the new rows but not the attention's output, and
-  // the attention only reads the buffers the compaction reads.  So the compress half runs on the handle's second,
-  // higher-priority stream beside the attention:
-  //   stream:  fork ........ append . fork' ........ attention ................................ join
-  //   side:         scores (diversity, norms) ....... [after fork'] selection, compaction ......./
+  // Scoring and selection (Eq. 5-8) read the cache and the new rows but not the attention's output, so they run on
+  // the handle's second, higher-priority stream beside the attention:
+  //   stream:  fork ........ append . fork' ........ attention ......................... join . [move]
+  //   side:         scores (diversity, norms) ....... [after fork'] selection [, gather] ..../
+  // The stable gather writes the other K/V buffer and stays on the side stream; the hole-filling move writes the
+  // buffer the attention reads and therefore follows the join on `stream`.
+  rc = validate_attend(h, layer, io);
+  if (rc) return rc;
   LayerState& S = h->layers[layer];
-  const ovggt_config& c = h->cfg;
+  const bool fill = fill_layout(h);
   CK(cudaEventRecord(h->ev_fork, st));
   CK(cudaStreamWaitEvent(h->side, h->ev_fork, 0));
-  if (c.score_mode == OVGGT_SCORE_HYBRID && S.n > 0 && S.colsum_nparts > 0 && io->frame_id > S.pending_frame) {
-    {
-      ProfScope ps(h, OVGGT_PROF_DIVERSITY, h->side);
-      rc = launch_diversity_from_parts(S.kbuf[S.cur], S.n, h->C, c.dtype, S.colsum_part, S.colsum_nparts, h->ksum,
-                                       S.d, io->resid, h->M, S.s_raw, h->side);
-    }
-    if (rc == OVGGT_OK) S.scores_frame = io->frame_id;
-  }
+  rc = enqueue_scores(h, S, io, h->side);
+  if (rc == OVGGT_OK) S.scores_frame = io->frame_id;
   if (rc == OVGGT_OK) rc = enqueue_append(h, layer, io, st);
   if (rc == OVGGT_OK) {
     CK(cudaEventRecord(h->ev_app, st));
     CK(cudaStreamWaitEvent(h->side, h->ev_app, 0));
     rc = enqueue_attention(h, layer, io, st);
   }
-  if (rc == OVGGT_OK) rc = ovggt_layer_compress(h, layer, io, h->side);
+  if (rc == OVGGT_OK) rc = compress_impl(h, layer, io, h->side, fill ? st : h->side);
   // join: whatever happened, the caller's stream is ordered after the side work
   S.scores_frame = -1;
   h->last_stream = st;
@@ -778,14 +941,30 @@ extern "C" int ovggt_cache_export(ovggt_cache* h, int32_t layer, int64_t* token_
   const LayerState& S = h->layers[layer];
   if (S.pending) return OVGGT_ERR_FRAME_ORDER;
   CK(cudaStreamSynchronize(h->last_stream));
-  const int n = S.n, b = S.cur;
+  const int n = S.n, b = S.cur, kb = S.kv;
   const size_t row = (size_t)h->C * h->elem;
   if (n > 0) {
     if (token_ids) CK(cudaMemcpy(token_ids, S.ids[b], (size_t)n * 8, cudaMemcpyDeviceToHost));
     if (flags) CK(cudaMemcpy(flags, S.flags[b], (size_t)n, cudaMemcpyDeviceToHost));
     if (scores) CK(cudaMemcpy(scores, S.stored[b], (size_t)n * 4, cudaMemcpyDeviceToHost));
-    if (k) CK(cudaMemcpy(k, S.kbuf[b], (size_t)n * row, cudaMemcpyDeviceToHost));
-    if (v) CK(cudaMemcpy(v, S.vbuf[b], (size_t)n * row, cudaMemcpyDeviceToHost));
+    if (!fill_layout(h)) {
+      if (k) CK(cudaMemcpy(k, S.kbuf[kb], (size_t)n * row, cudaMemcpyDeviceToHost));
+      if (v) CK(cudaMemcpy(v, S.vbuf[kb], (size_t)n * row, cudaMemcpyDeviceToHost));
+    } else if (k || v) {
+      // the rows lie in slot order on the device; the caller gets them in ascending token id
+      std::vector<int> slot(n);
+      std::vector<char> tmp((size_t)n * row);
+      CK(cudaMemcpy(slot.data(), S.slot[b], (size_t)n * 4, cudaMemcpyDeviceToHost));
+      for (int which = 0; which < 2; ++which) {
+        char* dst = static_cast<char*>(which == 0 ? k : v);
+        if (!dst) continue;
+        CK(cudaMemcpy(tmp.data(), which == 0 ? S.kbuf[kb] : S.vbuf[kb], (size_t)n * row, cudaMemcpyDeviceToHost));
+        for (int j = 0; j < n; ++j) {
+          if (slot[j] < 0 || slot[j] >= n) return OVGGT_ERR_DEVICE_STATUS;
+          std::memcpy(dst + (size_t)j * row, tmp.data() + (size_t)slot[j] * row, row);
+        }
+      }
+    }
   }
   if (n_out) *n_out = n;
   return OVGGT_OK;
@@ -824,17 +1003,23 @@ extern "C" int ovggt_cache_import(ovggt_cache* h, int32_t layer, const int64_t* 
     if (last_registration_frame != h->last_registration) return OVGGT_ERR_INVALID_ARG;
   }
   CK(cudaStreamSynchronize(h->last_stream));
-  const int b = S.cur;
+  const int b = S.cur, kb = S.kv;
   const size_t row = (size_t)h->C * h->elem;
   if (n > 0) {
     CK(cudaMemcpy(S.ids[b], token_ids, (size_t)n * 8, cudaMemcpyHostToDevice));
     CK(cudaMemcpy(S.flags[b], flags, (size_t)n, cudaMemcpyHostToDevice));
     CK(cudaMemcpy(S.stored[b], scores, (size_t)n * 4, cudaMemcpyHostToDevice));
-    CK(cudaMemcpy(S.kbuf[b], k, (size_t)n * row, cudaMemcpyHostToDevice));
-    CK(cudaMemcpy(S.vbuf[b], v, (size_t)n * row, cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(S.kbuf[kb], k, (size_t)n * row, cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(S.vbuf[kb], v, (size_t)n * row, cudaMemcpyHostToDevice));
+    if (fill_layout(h)) {         // rows arrive in token order: slot = position
+      std::vector<int> slot(n);
+      for (int j = 0; j < n; ++j) slot[j] = j;
+      CK(cudaMemcpy(S.slot[b], slot.data(), (size_t)n * 4, cudaMemcpyHostToDevice));
+    }
   }
   S.n = n;
   S.colsum_nparts = 0;          // the imported keys have not been summed
+  S.ksum_valid = false;
   S.pending = false;
   S.n_prot_init = n_init;
   S.n_prot_hist = n_hist;
@@ -862,6 +1047,8 @@ extern "C" int ovggt_cache_reset(ovggt_cache* h) {
     S.n_prot_init = S.n_prot_hist = 0;
     S.last_N = S.last_keep = 0;
     S.colsum_nparts = 0;
+    S.ksum_valid = false;
+    S.since_refresh = 0;
     S.scores_frame = -1;
   }
   h->anchors.clear();

@@ -137,12 +137,14 @@ __global__ void __launch_bounds__(1024) k_colsum_final_sliced(const float* __res
 }
 
 // d[row] = 1 - (k_row . ksum) / (|k_row| |ksum|); the cosine with the centroid equals the cosine
-// with the column sum.  A zero vector has cosine 0.  One warp per pair of rows; ksum is staged in shared memory
+// with the column sum.  ksum is given as n_slices rows of C floats that every CTA adds up in row order (one row: the
+// sums themselves; more: a base row plus corrections, as the hole-filling compaction leaves them).  A zero vector has cosine 0.  One warp per pair of rows; ksum is staged in shared memory
 // once per CTA and, for rows of up to 128 vectors, kept in registers by the lanes that meet its columns;
 // |ksum|^2 is folded by every warp in the same order, so all CTAs agree on it.
 template <int DT>
 __global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, int rows, int nvec,
                                                    const float* __restrict__ ksum, int n_slices,
+                                                   float* __restrict__ ksum_out,
                                                    float* __restrict__ d, int div_ctas,
                                                    const uint4* __restrict__ resid, int resid_rows,
                                                    float* __restrict__ s_raw) {
@@ -177,6 +179,7 @@ __global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, 
     float t = ksum[c];
     for (int sl = 1; sl < n_slices; ++sl) t += ksum[(size_t)sl * C + c];
     sh_ksum[c] = t;
+    if (ksum_out != nullptr && blockIdx.x == 0) ksum_out[c] = t;   // the folded sums, for whoever continues from them
   }
   __syncthreads();
   float kn = 0.0f;

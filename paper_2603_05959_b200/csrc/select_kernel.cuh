@@ -30,6 +30,8 @@ struct SelectShared {
   int pub_gt, pub_eq;        // this CTA's counts of keys above / equal to the threshold, read by the cluster
   float pub_lo_h, pub_hi_h, pub_lo_n, pub_hi_n;
   int all_gt[kSelectMaxCtas], all_eq[kSelectMaxCtas];   // the whole cluster's counts, gathered by one warp
+  int pub_up, pub_down;      // hole filling: survivors above the low range / evicted rows inside it, this CTA
+  int all_up[kSelectMaxCtas], all_down[kSelectMaxCtas];
   float mm[4];               // cluster-wide lo_h, hi_h, lo_n, hi_n
 };
 
@@ -232,11 +234,11 @@ __host__ __device__ inline size_t select_smem_bytes(int span, int np) {
          (size_t)np * 4 + (((size_t)np + 15) & ~(size_t)15) + 16;
 }
 
-// The fused per-step kernel also keeps the ids and stored scores of its positions (12 bytes each) and the frame's
-// raw residual norms (m floats) on chip.
+// The fused per-step kernel also keeps the ids, stored scores and physical slots of its positions (16 bytes each)
+// and the frame's raw residual norms (m floats) on chip.
 __host__ __device__ inline size_t compress_smem_bytes(int span, int np, int m) {
-  return select_smem_bytes(span, np) + (((size_t)span * 8 + 15) & ~(size_t)15) + (((size_t)span * 4 + 15) & ~(size_t)15) +
-         (((size_t)m * 4 + 15) & ~(size_t)15) + 16;
+  return select_smem_bytes(span, np) + (((size_t)span * 8 + 15) & ~(size_t)15) +
+         2 * (((size_t)span * 4 + 15) & ~(size_t)15) + (((size_t)m * 4 + 15) & ~(size_t)15) + 16;
 }
 
 // ---- standalone selection over given priorities: one cluster per independent problem (blockIdx.y)
@@ -279,7 +281,7 @@ struct CompressParams {
   int register_anchor, A;           // 1: flag the A most confident patches of the new frame HIST
   long long demote_frame;           // >= 0: release the HIST rows of that frame
   const float* s_raw;               // [M] residual norms of the new rows
-  const float* d;                   // [n] key diversity (hybrid mode)
+  const float* d;                   // key diversity (hybrid mode), indexed by the row's physical slot
   const float* conf;                // [grid_h*grid_w]
   const float* override_r;          // [N] or nullptr
   const long long* ids_src; const uint8_t* flags_src; const float* stored_src;   // [N] pre-compaction meta
@@ -288,6 +290,16 @@ struct CompressParams {
   int* survivors;                   // [min(N, B)]
   int* status;
   int* n_keep_out;
+  // Hole-filling layout (fill != 0): the K/V row of logical position g lives in slot slot_src[g] (g < n) or g
+  // (new rows); the K/V rows are not gathered.  Survivors whose slot is >= B have to move into the slots < B
+  // that evicted rows leave: the i-th such survivor (in logical order) goes to the i-th such slot (in the logical
+  // order of the rows that leave).  The kernel writes the pairs and the survivors' slots; the move kernel that
+  // follows copies the rows and patches slot_dst[move_j[i]] = move_dst[i].
+  int fill;
+  const int* slot_src;              // [n]
+  int* slot_dst;                    // [<= B]
+  int* move_src; int* move_dst; int* move_j;   // [<= M] each
+  int* n_moves_out;
 };
 
 // Eq. 6 for new-frame token j (aux tokens keep their raw score); s_raw: the frame's M residual norms.
@@ -330,7 +342,8 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
   unsigned char* q8 = smem + ((select_smem_bytes(span, Np) + 15) & ~(size_t)15);
   long long* sid = reinterpret_cast<long long*>(q8);              // [span] ids of the owned positions
   float* sst = reinterpret_cast<float*>(q8 + (((size_t)span * 8 + 15) & ~(size_t)15));   // [span] their stored scores
-  float* sraw = sst + (((size_t)span + 3) & ~(size_t)3);          // [M] the frame's residual norms
+  int* ssl = reinterpret_cast<int*>(sst + (((size_t)span + 3) & ~(size_t)3));   // [span] their physical slots
+  float* sraw = reinterpret_cast<float*>(ssl + (((size_t)span + 3) & ~(size_t)3)); // [M] the frame's residual norms
 
   // -- anchor registration (Sec. 3.3): the A most confident patch tokens of the new frame, ties to the lower
   //    index.  Every CTA computes the same marks and uses those of the positions it owns.
@@ -351,16 +364,25 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
     uint8_t f4[4];
     long long id4[4];
     float d4[4], st4[4];
+    int sl4[4];
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int i = i0 + u * nthr, g = begin + i;
+      sl4[u] = g;
       if (i < cnt) {
         f4[u] = P.flags_src[g];
         id4[u] = P.ids_src[g];
         if (g < n) {
           st4[u] = P.stored_src[g];
-          d4[u] = (P.mode == OVGGT_SCORE_HYBRID) ? P.d[g] : 0.0f;
+          if (P.fill) sl4[u] = P.slot_src[g];
         }
+      }
+    }
+    if (P.mode == OVGGT_SCORE_HYBRID) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * nthr, g = begin + i;
+        d4[u] = (i < cnt && g < n) ? P.d[sl4[u]] : 0.0f;
       }
     }
 #pragma unroll
@@ -384,6 +406,7 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
         val[i] = x;
         sid[i] = id4[u];
         sst[i] = keepscore;
+        ssl[i] = sl4[u];
       }
     }
   }
@@ -449,19 +472,22 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
   const int n_keep = cluster_select(cluster, keys, keep, begin, cnt, N, P.B, P.survivors, sh, &my_base, &bad);
 
   // -- compacted meta of this CTA's survivors (order preserved)
+  const int chunk = (cnt + nthr - 1) / nthr;
+  const int lo = min(cnt, tid * chunk), hi = min(cnt, lo + chunk);
+  int my_j;       // compacted index of this thread's first survivor
   {
-    const int chunk = (cnt + nthr - 1) / nthr;
-    const int lo = min(cnt, tid * chunk), hi = min(cnt, lo + chunk);
     int c = 0;
     for (int i = lo; i < hi; ++i) c += keep[i];
     int tot;
-    int j = my_base + block_excl_scan_int(c, sh->scan, &tot);
+    my_j = my_base + block_excl_scan_int(c, sh->scan, &tot);
+    int j = my_j;
     for (int i = lo; i < hi; ++i)
       if (keep[i]) {
         if (j < P.B) {
           P.ids_dst[j] = sid[i];
           P.flags_dst[j] = fl[i];
           P.stored_dst[j] = sst[i];
+          if (P.fill) P.slot_dst[j] = ssl[i];
         }
         ++j;
       }
@@ -469,6 +495,55 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
   if (rank == 0 && tid == 0) {
     *P.n_keep_out = n_keep;
     if (bad || n_keep != min(N, P.B)) atomicCAS(P.status, 0, OVGGT_ERR_DEVICE_STATUS);
+  }
+  if (P.fill) {
+    // -- hole filling: pair the survivors that sit above slot B with the slots below B whose rows leave
+    int up = 0, down = 0;
+    for (int i = lo; i < hi; ++i) {
+      up += keep[i] && ssl[i] >= P.B;
+      down += !keep[i] && ssl[i] < P.B;
+    }
+    int up_tot, down_tot;
+    int up_rank = block_excl_scan_int(up, sh->scan, &up_tot);
+    int down_rank = block_excl_scan_int(down, sh->scan, &down_tot);
+    if (tid == 0) {
+      sh->pub_up = up_tot;
+      sh->pub_down = down_tot;
+    }
+    cluster.sync();
+    if (tid < ncta) {
+      sh->all_up[tid] = *cluster.map_shared_rank(&sh->pub_up, tid);
+      sh->all_down[tid] = *cluster.map_shared_rank(&sh->pub_down, tid);
+    }
+    __syncthreads();
+    int up_all = 0, down_all = 0;
+    for (int r = 0; r < ncta; ++r) {
+      if (r < rank) {
+        up_rank += sh->all_up[r];
+        down_rank += sh->all_down[r];
+      }
+      up_all += sh->all_up[r];
+      down_all += sh->all_down[r];
+    }
+    int j = my_j;
+    for (int i = lo; i < hi; ++i) {
+      if (keep[i]) {
+        if (ssl[i] >= P.B && up_rank < M) {
+          P.move_src[up_rank] = ssl[i];
+          P.move_j[up_rank] = j;
+          ++up_rank;
+        }
+        ++j;
+      } else if (ssl[i] < P.B && down_rank < M) {
+        P.move_dst[down_rank++] = ssl[i];
+      }
+    }
+    if (rank == 0 && tid == 0) {
+      // the two counts agree whenever the slots below min(N, B) were all occupied, which the layout guarantees
+      const bool consistent = up_all == down_all && up_all <= M;
+      *P.n_moves_out = consistent ? up_all : 0;
+      if (!consistent) atomicCAS(P.status, 0, OVGGT_ERR_DEVICE_STATUS);
+    }
   }
   cluster.sync();   // no CTA may exit while others still read its shared memory
 }

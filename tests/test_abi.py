@@ -39,13 +39,13 @@ def test_library_exports_every_declared_symbol(lib):
 def _cfg(**over):
     kw = dict(n_layers=1, n_heads=4, head_dim=64, n_special=5, grid_h=8, grid_w=8, budget=256,
               anchor_tokens=8, k_max=3, min_anchor_interval=4, tau=0.2, alpha=0.5, beta=0.5,
-              protect_first_frame=1, score_mode=0, dtype=0)
+              protect_first_frame=1, score_mode=0, dtype=0, compaction=1)
     kw.update(over)
     budgets = (C.c_int32 * kw["n_layers"])(*([kw.pop("budget")] * kw["n_layers"]))
     cfg = B.OvggtConfig(kw["n_layers"], kw["n_heads"], kw["head_dim"], kw["n_special"], kw["grid_h"],
                         kw["grid_w"], budgets, kw["anchor_tokens"], kw["k_max"], kw["min_anchor_interval"],
                         kw["tau"], kw["alpha"], kw["beta"], kw["protect_first_frame"], kw["score_mode"],
-                        kw["dtype"], None, 0)
+                        kw["dtype"], kw["compaction"], None, 0)
     cfg._keep = budgets
     return cfg
 
@@ -54,7 +54,9 @@ def test_workspace_bytes_is_a_pure_host_function(lib):
     cfg = _cfg()
     need = lib.ovggt_workspace_bytes(C.byref(cfg))
     M, Cdim, R = 69, 256, 256 + 69
-    assert need >= 4 * R * Cdim * 4              # two K and two V buffers of B + M rows, fp32
+    assert need >= 4 * R * Cdim * 4              # stable gather: two K and two V buffers of B + M rows, fp32
+    holes = lib.ovggt_workspace_bytes(C.byref(_cfg(compaction=0)))
+    assert 2 * R * Cdim * 4 <= holes < need      # hole filling: one K and one V buffer
     big = lib.ovggt_workspace_bytes(C.byref(_cfg(budget=512)))
     assert big > need
     # the bf16 VGGT-shaped layer: 2 x 2 x (16384 + 1374) x 1024 x 2 bytes of K/V
@@ -66,7 +68,7 @@ def test_workspace_bytes_is_a_pure_host_function(lib):
 def test_create_reports_config_errors_without_a_gpu(lib):
     h = C.c_void_p()
     bad = [(_cfg(head_dim=32), -1), (_cfg(n_layers=0, budget=256), -1), (_cfg(dtype=7), -1),
-           (_cfg(alpha=1.5), -1), (_cfg(k_max=17), -1), (_cfg(anchor_tokens=65), -1),
+           (_cfg(alpha=1.5), -1), (_cfg(k_max=17), -1), (_cfg(anchor_tokens=65), -1), (_cfg(compaction=2), -1),
            (_cfg(budget=68), -3), (_cfg(budget=69 + 3 * 8 - 1), -3)]
     for cfg, code in bad:
         assert lib.ovggt_workspace_bytes(C.byref(cfg)) == 0

@@ -41,6 +41,42 @@ def test_two_gloo_ranks_take_the_slowest_time_and_add_the_frames():
     assert replicas.max_over_ranks([3.0], 1) == [3.0]      # a single rank needs no process group
 
 
+def test_gpus_flag_alone_starts_the_ranks():
+    """`python bench.py --gpus 2` with no launcher around it must start two ranks itself.  The launch-check arm goes
+    through the same spawner as the GPU arm and reports, over gloo, what the ranks saw."""
+    import json
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "launch-check"],
+                       env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["local_ranks_plus_one"] == [1, 2]
+    assert lines[0]["max_over_ranks_ms"] == 11.0 and lines[0]["master_addr"] == "127.0.0.1"
+
+
+def test_clock_sampler_tags_phases_and_survives_a_region_shorter_than_its_period():
+    sys.path.insert(0, ROOT)
+    import bench
+    rows = bench.ClockSampler.parse_rows([
+        "2026/01/01 00:00:00.010, 1965, 1965, 300.0, 0x0, Not Active, Not Active, Not Active, Not Active",
+        "2026/01/01 00:00:01.000, 1800, 1965, 900.0, 0x4, Not Active, Not Active, Not Active, Active",
+        "2026/01/01 00:00:01.020, 1790, 1965, 950.0, 0x4, Not Active, Not Active, Not Active, Active",
+        "garbage"])
+    assert len(rows) == 3 and rows[1][4] == ["sw_power_cap"]
+    import datetime
+    t = lambda s: datetime.datetime.strptime(s, "%Y/%m/%d %H:%M:%S.%f").timestamp()
+    marks = [(t("2026/01/01 00:00:00.000"), "setup"), (t("2026/01/01 00:00:00.900"), "warmup"),
+             (t("2026/01/01 00:00:01.015"), "timed"), (t("2026/01/01 00:00:01.050"), "after")]
+    res = bench.ClockSampler.summarise(rows, marks, t("2026/01/01 00:00:02.000"))
+    assert res["samples_in_timed_region"] == 1 and res["sm_mhz"] == 1790.0 and res["reasons"] == ["sw_power_cap"]
+    # no sample inside the timed region: the samples under load stand in, the set-up phase does not
+    marks[2] = (t("2026/01/01 00:00:01.040"), "timed")
+    res = bench.ClockSampler.summarise(rows, marks, t("2026/01/01 00:00:02.000"))
+    assert res["samples_in_timed_region"] == 0 and res["samples"] == 2 and res["sm_mhz"] == 1795.0
+    assert res["phases"]["setup"]["sm_mhz"] == 1965.0
+
+
 def test_reference_arm_runs_on_rank_zero_only():
     env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
