@@ -21,7 +21,7 @@ class OrcConfig(C.Structure):
         ("k_max", C.c_int32), ("min_anchor_interval", C.c_int32),
         ("tau", C.c_double), ("alpha", C.c_double), ("beta", C.c_double),
         ("protect_first_frame", C.c_int32), ("score_mode", C.c_int32),
-        ("diversity_per_head", C.c_int32),
+        ("diversity_per_head", C.c_int32), ("camera_cache", C.c_int32),
     ]
 
 
@@ -54,6 +54,9 @@ def lib():
         L.orc_compress.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_double,
                                    C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_int32),
                                    C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int64)]
+        L.orc_compress_camera.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.c_int32, C.c_int64,
+                                          C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_int32),
+                                          C.POINTER(C.c_int32)]
         L.orc_export.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_uint8),
                                  C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_float)]
         L.orc_residual_norms.argtypes = [C.POINTER(C.c_float), C.c_int32, C.c_int32, C.POINTER(C.c_double)]
@@ -162,10 +165,10 @@ class OracleLayer:
 
     def __init__(self, *, n_heads, head_dim, n_special, grid_h, grid_w, budget, anchor_tokens,
                  k_max=3, min_anchor_interval=100, tau=0.2, alpha=0.5, beta=0.5,
-                 protect_first_frame=1, score_mode=0, diversity_per_head=0):
+                 protect_first_frame=1, score_mode=0, diversity_per_head=0, camera_cache=0):
         self.cfg = OrcConfig(n_heads, head_dim, n_special, grid_h, grid_w, budget, anchor_tokens,
                              k_max, min_anchor_interval, tau, alpha, beta, protect_first_frame,
-                             score_mode, diversity_per_head)
+                             score_mode, diversity_per_head, camera_cache)
         self.M = n_special + grid_h * grid_w
         self.C = n_heads * head_dim
         self._h = lib().orc_create(C.byref(self.cfg))
@@ -242,6 +245,28 @@ class OracleLayer:
             raise RuntimeError(f"orc_compress failed: {rc}")
         return {"r": r, "survivors": surv[: n_s.value].copy(), "registered": bool(reg.value),
                 "demoted_frame": int(dem.value)}
+
+    def compress_camera(self, resid, registered=False, demoted_frame=-1, score_override=None):
+        """Supp. C: compress step of the camera head's cache; the anchor decision comes from the aggregator."""
+        resid = _f32(resid)
+        assert resid.shape == (1, self.C)
+        N = self.n_rows
+        ov = None if score_override is None else _f32(score_override)
+        r = np.empty(N, dtype=np.float32)
+        surv = np.empty(N, dtype=np.int32)
+        n_s = C.c_int32(0)
+        rc = lib().orc_compress_camera(self._h, _ptr(resid, C.c_float), int(bool(registered)), int(demoted_frame),
+                                       _ptr(ov, C.c_float), _ptr(r, C.c_float), _ptr(surv, C.c_int32), C.byref(n_s))
+        if rc != 0:
+            raise RuntimeError(f"orc_compress_camera failed: {rc}")
+        return {"r": r, "survivors": surv[: n_s.value].copy()}
+
+    @classmethod
+    def camera(cls, *, n_heads, head_dim, budget, k_max=3, beta=0.5, protect_first_frame=1, score_mode=0):
+        """The camera head's cache: one token per frame (Supp. C)."""
+        return cls(n_heads=n_heads, head_dim=head_dim, n_special=1, grid_h=0, grid_w=0, budget=budget,
+                   anchor_tokens=0, k_max=k_max, beta=beta, protect_first_frame=protect_first_frame,
+                   score_mode=score_mode, camera_cache=1)
 
     def export(self, with_kv=True):
         n = self.n_rows

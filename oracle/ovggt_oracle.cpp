@@ -95,7 +95,7 @@ extern "C" void orc_diversity(const float* K, int32_t n, int32_t C, int32_t n_he
 
 /* ------------------------------------------------------------------ Eq. 7 */
 static void minmax_group(const double* x, const uint8_t* flags, int32_t count, double weight,
-                         float* r) {
+                         float* r, double lone_value = 0.0) {
   double lo = std::numeric_limits<double>::infinity(), hi = -lo;
   int32_t members = 0;
   for (int32_t i = 0; i < count; ++i)
@@ -109,6 +109,7 @@ static void minmax_group(const double* x, const uint8_t* flags, int32_t count, d
       r[i] = std::numeric_limits<float>::infinity();
     } else {
       double hat = (members > 0 && hi > lo) ? (x[i] - lo) / (hi - lo) : 0.0;
+      if (members == 1) hat = lone_value;   /* 0/0: a reading, 0 for the aggregator, 1 for the camera cache */
       r[i] = (float)(weight * hat);
     }
   }
@@ -211,13 +212,20 @@ struct orc_state {
 };
 
 extern "C" orc_state* orc_create(const orc_config* cfg) {
-  if (!cfg || cfg->n_heads < 1 || cfg->head_dim < 1 || cfg->n_special < 0 || cfg->grid_h < 1 ||
-      cfg->grid_w < 1 || cfg->anchor_tokens < 0 || cfg->k_max < 0 ||
-      cfg->anchor_tokens > cfg->grid_h * cfg->grid_w)
+  if (!cfg || cfg->n_heads < 1 || cfg->head_dim < 1 || cfg->n_special < 0 || cfg->anchor_tokens < 0 ||
+      cfg->k_max < 0)
     return nullptr;
+  if (cfg->camera_cache) {
+    /* Supp. C: one camera token per frame, nothing else */
+    if (cfg->n_special != 1 || cfg->grid_h != 0 || cfg->grid_w != 0 || cfg->anchor_tokens != 0) return nullptr;
+  } else if (cfg->grid_h < 1 || cfg->grid_w < 1 || cfg->anchor_tokens > cfg->grid_h * cfg->grid_w) {
+    return nullptr;
+  }
   const int64_t M = cfg->n_special + (int64_t)cfg->grid_h * cfg->grid_w;
-  /* Eq. 9: the protected set can reach M + K_max * A; the budget must hold it. */
-  const int64_t pmax = (cfg->protect_first_frame ? M : 0) + (int64_t)cfg->k_max * cfg->anchor_tokens;
+  /* Eq. 9: the protected set can reach M + K_max * A; the budget must hold it.  (Camera cache: an anchor is the
+   * frame's one token.) */
+  const int64_t per_anchor = cfg->camera_cache ? 1 : cfg->anchor_tokens;
+  const int64_t pmax = (cfg->protect_first_frame ? M : 0) + (int64_t)cfg->k_max * per_anchor;
   if (cfg->budget < M || cfg->budget < pmax) return nullptr;
   orc_state* st = new orc_state();
   st->cfg = *cfg;
@@ -275,6 +283,36 @@ extern "C" int orc_attend(orc_state* st, int64_t frame_id, const float* q, const
   return 0;
 }
 
+/* Budgeted retention (Eq. 8) and order-preserving compaction, given the priorities r [N]. */
+static int select_and_compact(orc_state* st, const std::vector<float>& r, int32_t* survivors,
+                              int32_t* n_survivors) {
+  const int32_t C = st->C, N = (int32_t)st->ids.size();
+  std::vector<int32_t> keep(N);
+  int32_t n_keep = 0;
+  if (orc_select(r.data(), st->flags.data(), N, st->cfg.budget, keep.data(), &n_keep) != 0) return -4;
+  std::vector<int64_t> ids(n_keep);
+  std::vector<uint8_t> flags(n_keep);
+  std::vector<float> stored(n_keep), kk((size_t)n_keep * C), vv((size_t)n_keep * C);
+  for (int32_t j = 0; j < n_keep; ++j) {
+    const int32_t src = keep[j];
+    ids[j] = st->ids[src];
+    flags[j] = st->flags[src];
+    stored[j] = st->stored[src];
+    std::memcpy(&kk[(size_t)j * C], &st->k[(size_t)src * C], sizeof(float) * C);
+    std::memcpy(&vv[(size_t)j * C], &st->v[(size_t)src * C], sizeof(float) * C);
+  }
+  st->evicted_total += N - n_keep;
+  st->ids.swap(ids);
+  st->flags.swap(flags);
+  st->stored.swap(stored);
+  st->k.swap(kk);
+  st->v.swap(vv);
+  st->pending = false;
+  if (survivors) std::memcpy(survivors, keep.data(), sizeof(int32_t) * n_keep);
+  if (n_survivors) *n_survivors = n_keep;
+  return 0;
+}
+
 extern "C" int orc_compress(orc_state* st, const float* resid, const float* conf, double rho,
                             const float* score_override, float* r_out, int32_t* survivors,
                             int32_t* n_survivors, int32_t* registered, int64_t* demoted_frame) {
@@ -329,33 +367,63 @@ extern "C" int orc_compress(orc_state* st, const float* resid, const float* conf
       if (st->flags[i] == ORC_FLAG_EVICTABLE) r[i] = score_override[i];
   if (r_out) std::memcpy(r_out, r.data(), sizeof(float) * N);
 
-  /* Budgeted retention (Eq. 8) and order-preserving compaction. */
-  std::vector<int32_t> keep(N);
-  int32_t n_keep = 0;
-  if (orc_select(r.data(), st->flags.data(), N, cfg.budget, keep.data(), &n_keep) != 0) return -4;
-  std::vector<int64_t> ids(n_keep);
-  std::vector<uint8_t> flags(n_keep);
-  std::vector<float> stored(n_keep), kk((size_t)n_keep * C), vv((size_t)n_keep * C);
-  for (int32_t j = 0; j < n_keep; ++j) {
-    const int32_t src = keep[j];
-    ids[j] = st->ids[src];
-    flags[j] = st->flags[src];
-    stored[j] = st->stored[src];
-    std::memcpy(&kk[(size_t)j * C], &st->k[(size_t)src * C], sizeof(float) * C);
-    std::memcpy(&vv[(size_t)j * C], &st->v[(size_t)src * C], sizeof(float) * C);
-  }
-  st->evicted_total += N - n_keep;
-  st->ids.swap(ids);
-  st->flags.swap(flags);
-  st->stored.swap(stored);
-  st->k.swap(kk);
-  st->v.swap(vv);
-  st->pending = false;
-  if (survivors) std::memcpy(survivors, keep.data(), sizeof(int32_t) * n_keep);
-  if (n_survivors) *n_survivors = n_keep;
+  int rc = select_and_compact(st, r, survivors, n_survivors);
+  if (rc != 0) return rc;
   if (registered) *registered = did_register;
   if (demoted_frame) *demoted_frame = demoted;
   return 0;
+}
+
+/* ------------------------------------------------------------------ Supp. C: the camera head's cache */
+extern "C" int orc_compress_camera(orc_state* st, const float* resid, int32_t registered,
+                                   int64_t demoted_frame, const float* score_override, float* r_out,
+                                   int32_t* survivors, int32_t* n_survivors) {
+  if (!st->pending) return -2;
+  const orc_config& cfg = st->cfg;
+  if (!cfg.camera_cache || st->M != 1) return -5;
+  const int32_t C = st->C;
+  const int32_t N = (int32_t)st->ids.size(), n = N - 1;
+  const int64_t t = st->last_frame;
+
+  /* Activation Value Rating (Eq. 5) of the frame's one token; there is no map to smooth (Eq. 6 does not apply). */
+  double s = 0.0;
+  orc_residual_norms(resid, 1, C, &s);
+  st->stored[n] = (float)s;
+
+  /* Protection follows the aggregator's decision for this frame (Sec. 3.3 applied there, mirrored here). */
+  if (t == st->first_frame) {
+    if (cfg.protect_first_frame) st->flags[n] = ORC_FLAG_INIT;
+  } else if (registered) {
+    st->flags[n] = ORC_FLAG_HIST;
+    st->anchors.push_back(t);
+    st->last_registration = t;
+  }
+  if (demoted_frame >= 0) {
+    for (int32_t i = 0; i < N; ++i)
+      if (st->flags[i] == ORC_FLAG_HIST && st->ids[i] == demoted_frame) st->flags[i] = ORC_FLAG_EVICTABLE;
+    for (auto it = st->anchors.begin(); it != st->anchors.end(); ++it)
+      if (*it == demoted_frame) {
+        st->anchors.erase(it);
+        break;
+      }
+  }
+
+  std::vector<float> r(N);
+  if (cfg.score_mode == ORC_SCORE_HYBRID) {
+    std::vector<double> d(std::max(n, 1));
+    orc_diversity(st->k.data(), n, C, cfg.n_heads, cfg.diversity_per_head, d.data());
+    minmax_group(d.data(), st->flags.data(), n, 1.0 - cfg.beta, r.data());
+    minmax_group(&s, st->flags.data() + n, 1, cfg.beta, r.data() + n, /*lone_value=*/1.0);
+  } else {
+    for (int32_t i = 0; i < N; ++i)
+      r[i] = st->flags[i] != ORC_FLAG_EVICTABLE ? std::numeric_limits<float>::infinity()
+                                                : st->stored[i];
+  }
+  if (score_override)
+    for (int32_t i = 0; i < N; ++i)
+      if (st->flags[i] == ORC_FLAG_EVICTABLE) r[i] = score_override[i];
+  if (r_out) std::memcpy(r_out, r.data(), sizeof(float) * N);
+  return select_and_compact(st, r, survivors, n_survivors);
 }
 
 extern "C" void orc_export(const orc_state* st, int64_t* ids, uint8_t* flags, float* stored,

@@ -17,7 +17,8 @@
  * selection against a brute-force sort, smoothing / diversity / min-max
  * against closed forms and special cases, anchor FIFO against a hand-written
  * schedule, the budget and protected-size invariants (Eq. 8, Eq. 9), and the
- * full-cache footprint formula of Sec. 3.1.
+ * full-cache footprint formula of Sec. 3.1; the camera-head cache against the aggregator's anchor schedule and
+ * closed forms of its two differences.
  * Parity unpinned: the reconstruction accuracy the paper reports for the
  * method (needs its datasets and trained weights).
  */
@@ -43,6 +44,7 @@ typedef struct {
   int32_t protect_first_frame;           /* Global Initial Anchor on/off */
   int32_t score_mode;                    /* ORC_SCORE_* */
   int32_t diversity_per_head;            /* 0: cosine on the whole C-vector; 1: mean over heads of per-head cosine */
+  int32_t camera_cache;                  /* 1: the camera head's cache (Supp. C): one token per frame, grid 0 x 0 */
 } orc_config;
 
 typedef struct orc_state orc_state;
@@ -109,6 +111,18 @@ int orc_attend(orc_state* st, int64_t frame_id, const float* q, const float* k, 
 int orc_compress(orc_state* st, const float* resid, const float* conf, double rho,
                  const float* score_override, float* r_out, int32_t* survivors,
                  int32_t* n_survivors, int32_t* registered, int64_t* demoted_frame);
+
+/* Supp. C: the camera prediction head keeps one token per frame in a cache of its own, managed by the same scoring
+ * and protection with two differences: there is no patch map, hence no smoothing (the stored score is the raw
+ * residual norm), and the anchor flags are not decided here but follow the aggregator's decision for the same frame:
+ * registered != 0 protects this frame's token as a historical anchor, demoted_frame >= 0 releases that frame's token.
+ * Eq. 7's min-max of the new group has a single member (0/0): its normalised score is taken as 1, so the token ranks
+ * at beta (with 0 it would tie with the least diverse cached token, lose by position and never enter the cache).
+ * For a state created with camera_cache = 1 (n_special = 1, grid 0 x 0, anchor_tokens 0; the budget must hold
+ * 1 + k_max tokens).  Other arguments as orc_compress. */
+int orc_compress_camera(orc_state* st, const float* resid, int32_t registered, int64_t demoted_frame,
+                        const float* score_override, float* r_out, int32_t* survivors,
+                        int32_t* n_survivors);
 
 /* Current layout, ascending token id.  Any pointer may be NULL. */
 void orc_export(const orc_state* st, int64_t* ids, uint8_t* flags, float* stored, float* k, float* v);

@@ -428,6 +428,79 @@ def test_stored_scores_travel_with_their_rows_through_every_compaction():
     assert len({int(i) // M for i in layer.export(with_kv=False)["ids"]}) >= 3
 
 
+# ------------------------------------------------------------------ Supp. C: the camera head's cache
+
+def _camera_token(cfg, t, tag):
+    """One seeded row of `cfg.dim` values for frame t (the camera token's q, k, v or residual)."""
+    rng = np.random.Generator(np.random.Philox(key=[np.uint64(cfg.seed + 77), np.uint64((t << 8) | tag)]))
+    return gen.round_to_dtype(rng.standard_normal((1, cfg.dim), dtype=np.float32) * (1.0 + 0.1 * tag), cfg.dtype)
+
+
+def test_camera_cache_follows_the_aggregators_anchor_schedule():
+    """One token per frame under the same scoring and protection (Supp. C).  The aggregator oracle runs a stream with
+    frequent anchor turnover; its decision of each frame (registered, demoted frame) drives the camera cache.  The
+    camera cache's protected tokens must be exactly the first frame and the aggregator's active anchors after every
+    frame, never be evicted while active, and the cache must hold min(t + 1, B_cam) tokens."""
+    cfg = gen.config_tiny().replace(tau=0.95, min_anchor_interval=2, k_max=2, n_frames=30)
+    agg = orc.OracleLayer.from_stream(cfg)
+    cam = orc.OracleLayer.camera(n_heads=cfg.n_heads, head_dim=cfg.head_dim, budget=7, k_max=cfg.k_max)
+    demotions = 0
+    for t in range(cfg.n_frames):
+        fi = gen.frame_inputs(cfg, t)
+        agg.attend(t, fi.q, fi.k, fi.v, compute=False)
+        dec = agg.compress(fi.resid, fi.conf, fi.rho)
+        demotions += dec["demoted_frame"] >= 0
+        cam.attend(t, _camera_token(cfg, t, 1), _camera_token(cfg, t, 2), _camera_token(cfg, t, 3), compute=False)
+        cam.compress_camera(_camera_token(cfg, t, 4), dec["registered"], dec["demoted_frame"])
+        ex = cam.export(with_kv=False)
+        assert len(ex["ids"]) == min(t + 1, 7) and np.all(np.diff(ex["ids"]) > 0)
+        assert ex["ids"][0] == 0 and ex["flags"][0] == 1                       # the first frame's token, for good
+        assert sorted(ex["ids"][ex["flags"] == 2].tolist()) == agg.anchors()   # the same anchors, token for token
+        assert cam.anchors() == agg.anchors()
+    assert demotions >= 3 and len(agg.anchors()) == 2
+
+
+def test_camera_cache_scores_closed_forms():
+    """No smoothing: the stored score is the raw residual norm.  The lone new token ranks at beta exactly; cached
+    tokens at (1 - beta) x the min-max of their cosine distances to the centroid key (library cosine)."""
+    C, H = 128, 2
+    cam = orc.OracleLayer.camera(n_heads=H, head_dim=64, budget=5, beta=0.3, protect_first_frame=0)
+    rng = np.random.default_rng(8)
+    keys, norms = [], []
+    for t in range(9):
+        q, k, v, r = (rng.standard_normal((1, C)).astype(np.float32) for _ in range(4))
+        keys.append(k[0]); norms.append(np.float32(np.linalg.norm(r.astype(np.float64))))
+        cam.attend(t, q, k, v, compute=False)
+        pre = cam.export(with_kv=False)
+        out = cam.compress_camera(r)
+        n = len(pre["ids"]) - 1
+        assert out["r"][n] == np.float32(0.3)                                   # beta x 1
+        if n >= 2:
+            K = np.stack([keys[int(i)] for i in pre["ids"][:n]]).astype(np.float64)
+            d = np.array([scipy.spatial.distance.cosine(k_, K.mean(0)) for k_ in K])
+            want = 0.7 * (d - d.min()) / (d.max() - d.min())
+            np.testing.assert_allclose(out["r"][:n], want, rtol=0, atol=1e-6)
+            # Eq. 8 by brute force: the budget's worth of largest priorities, ties to the lower position
+            order = sorted(range(n + 1), key=lambda i: (-out["r"][i], i))[:5]
+            np.testing.assert_array_equal(out["survivors"], sorted(order))
+        ex = cam.export(with_kv=False)
+        np.testing.assert_array_equal(ex["stored"], [norms[int(i)] for i in ex["ids"]])
+    assert cam.evicted_total == 4
+
+
+def test_camera_cache_config_rules():
+    with pytest.raises(ValueError):                       # the budget must hold the first frame and K_max anchors
+        orc.OracleLayer.camera(n_heads=1, head_dim=8, budget=3, k_max=3)
+    orc.OracleLayer.camera(n_heads=1, head_dim=8, budget=4, k_max=3).close()
+    with pytest.raises(ValueError):                       # a camera cache has no patch grid
+        orc.OracleLayer(n_heads=1, head_dim=8, n_special=1, grid_h=2, grid_w=2, budget=16, anchor_tokens=0, camera_cache=1)
+    agg = _tiny_layer()
+    x = np.zeros((agg.M, agg.C), np.float32)
+    agg.attend(0, x, x, x, compute=False)
+    with pytest.raises(RuntimeError):                     # and the aggregator's cache is not a camera cache
+        agg.compress_camera(np.zeros((1, agg.C), np.float32))
+
+
 def test_create_rejects_budget_below_protected_bound():
     with pytest.raises(ValueError):
         _tiny_layer(budget=14 + 2 * 3 - 1)          # M + K_max * A = 20
