@@ -83,6 +83,8 @@ typedef struct {
   int32_t score_mode;                    /* OVGGT_SCORE_HYBRID (Eq. 7) or OVGGT_SCORE_RESIDUAL_STORED */
   int32_t dtype;                         /* OVGGT_DTYPE_* of q, k, v, resid, out and of the cache */
   int32_t compaction;                    /* OVGGT_COMPACT_* */
+  int32_t camera_head;                   /* 1: the camera head's cache (Supp. C): n_special = 1, grid 0 x 0,
+                                            anchor_tokens = 0; see ovggt_camera_compress.  0: an aggregator cache */
   void* workspace;                       /* device, >= ovggt_workspace_bytes(cfg), 1024-byte aligned; need not be zeroed */
   size_t workspace_bytes;
 } ovggt_config;
@@ -140,6 +142,20 @@ int ovggt_layer_attend(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* 
  * score_override. */
 int ovggt_layer_compress(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
 
+/* Supp. C: the camera prediction head keeps one token per frame in a cache of its own, under the same scoring and
+ * protection.  Create it as a second handle with camera_head = 1 (budget[l] >= 1 + K_max tokens), run
+ * ovggt_layer_attend on it with the camera token's q, k, v ([1, C]), and compress it with this call instead of
+ * ovggt_layer_compress.  Differences from the aggregator's cache: no patch map, hence no smoothing (Eq. 6 does not
+ * apply; the stored score is the raw residual norm); the anchor flags are not decided from rho but mirror the
+ * aggregator's decision for the same frame_id - registered != 0 protects this frame's token, demoted_frame >= 0
+ * releases that frame's token; the new group of Eq. 7 has one member (0/0), whose normalised score is taken as 1.
+ * ovggt_cache_anchor_decision reads (registered, demoted_frame) of frame_id from the aggregator handle once one of
+ * its layers has compressed that frame (OVGGT_ERR_FRAME_ORDER before that, or once a later frame was decided).
+ * Uses frame_id, resid ([1, C]), score_override of io. */
+int ovggt_cache_anchor_decision(ovggt_cache* aggregator, int64_t frame_id, int32_t* registered, int64_t* demoted_frame);
+int ovggt_camera_compress(ovggt_cache* camera, int32_t layer, const ovggt_frame_io* io, int32_t registered,
+                          int64_t demoted_frame, void* stream);
+
 /* ovggt_layer_attend and ovggt_layer_compress of one (frame, layer): the whole hot path.  Scoring and selection
  * read the cache and the new rows but not the attention's output, so they are enqueued on a second stream that the
  * handle owns (a host object, created by ovggt_cache_create), forked from and joined back into `stream` with
@@ -187,6 +203,17 @@ int ovggt_cache_import(ovggt_cache* cache, int32_t layer, const int64_t* token_i
 
 /* Forget every frame: all layers empty, no anchors, no first frame, device status cleared.  Synchronises. */
 int ovggt_cache_reset(ovggt_cache* cache);
+
+/* Every device-side wait of the library (the attention kernel waits on shared-memory barriers for its bulk copies
+ * and tensor-core instructions) is bounded: when it runs out, the kernel returns cleanly and leaves OVGGT_ERR_TIMEOUT
+ * in the handle's device status word, which ovggt_cache_stats reports and which stays set until cleared.
+ * ovggt_cache_selftest_bounded_wait exercises exactly that wait routine on the GPU without any copy or tensor-core
+ * work: one warp waits, for at most limit_us microseconds (1 .. 1,000,000), on a barrier that nothing will ever
+ * complete.  Afterwards the status word holds OVGGT_ERR_TIMEOUT; *waited_ns (host, may be NULL; non-NULL
+ * synchronises) is how long the wait lasted.  ovggt_cache_clear_status zeroes the status word (synchronises), after
+ * which the handle is used as before. */
+int ovggt_cache_selftest_bounded_wait(ovggt_cache* cache, uint32_t limit_us, uint64_t* waited_ns, void* stream);
+int ovggt_cache_clear_status(ovggt_cache* cache);
 
 /* Results of the layer's last compress, copied to host (each pointer may be NULL): priorities [N] as the
  * library computed them (+inf on protected rows; its own values even when score_override was ranked instead),

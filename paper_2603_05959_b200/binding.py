@@ -25,7 +25,8 @@ PROF_CLASSES = ["append", "attention", "row_norms", "diversity", "select", "comp
 EXPORTED = [
     "ovggt_workspace_bytes", "ovggt_cache_create", "ovggt_cache_destroy", "ovggt_layer_attend",
     "ovggt_layer_compress", "ovggt_layer_step", "ovggt_layer_step_host", "ovggt_cache_stats",
-    "ovggt_cache_export", "ovggt_cache_import", "ovggt_cache_reset", "ovggt_cache_last_selection", "ovggt_kernel_launches",
+    "ovggt_cache_export", "ovggt_cache_import", "ovggt_cache_reset", "ovggt_cache_anchor_decision",
+    "ovggt_camera_compress", "ovggt_cache_selftest_bounded_wait", "ovggt_cache_clear_status", "ovggt_cache_last_selection", "ovggt_kernel_launches",
     "ovggt_cache_profile_enable", "ovggt_cache_profile_read", "ovggt_cache_set_overlap",
     "ovggt_strerror", "ovggt_last_cuda_error", "ovggt_k_row_norms", "ovggt_k_diversity_scratch_bytes",
     "ovggt_k_diversity", "ovggt_k_diversity_static", "ovggt_k_select", "ovggt_k_compact", "ovggt_k_attention_scratch_bytes",
@@ -41,7 +42,7 @@ class OvggtConfig(C.Structure):
         ("anchor_tokens", C.c_int32), ("k_max", C.c_int32), ("min_anchor_interval", C.c_int32),
         ("tau", C.c_float), ("alpha", C.c_float), ("beta", C.c_float),
         ("protect_first_frame", C.c_int32), ("score_mode", C.c_int32), ("dtype", C.c_int32),
-        ("compaction", C.c_int32),
+        ("compaction", C.c_int32), ("camera_head", C.c_int32),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
     ]
 
@@ -94,6 +95,10 @@ def lib():
         L.ovggt_cache_export.argtypes = [vp, i32, vp, vp, vp, vp, vp, C.POINTER(i32)]
         L.ovggt_cache_import.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32, i64, i64]
         L.ovggt_cache_reset.argtypes = [vp]
+        L.ovggt_cache_clear_status.argtypes = [vp]
+        L.ovggt_cache_selftest_bounded_wait.argtypes = [vp, C.c_uint32, C.POINTER(C.c_uint64), vp]
+        L.ovggt_cache_anchor_decision.argtypes = [vp, i64, C.POINTER(i32), C.POINTER(i64)]
+        L.ovggt_camera_compress.argtypes = [vp, i32, C.POINTER(OvggtFrameIO), i32, i64, vp]
         L.ovggt_cache_last_selection.argtypes = [vp, i32, vp, C.POINTER(i32), vp, C.POINTER(i32)]
         L.ovggt_cache_profile_enable.argtypes = [vp, i32]
         L.ovggt_cache_set_overlap.argtypes = [vp, i32]
@@ -152,13 +157,13 @@ class OvggtCache:
     def __init__(self, *, n_layers=1, n_heads=16, head_dim=64, n_special=5, grid_h=37, grid_w=37,
                  budget=16384, anchor_tokens=64, k_max=3, min_anchor_interval=100, tau=0.2, alpha=0.5,
                  beta=0.5, protect_first_frame=1, score_mode=SCORE_HYBRID, dtype=DTYPE_BF16,
-                 compaction=COMPACT_FILL_HOLES, device: Optional[torch.device] = None):
+                 compaction=COMPACT_FILL_HOLES, camera_head=0, device: Optional[torch.device] = None):
         budgets = [budget] * n_layers if isinstance(budget, int) else list(budget)
         assert len(budgets) == n_layers
         self._budgets = (C.c_int32 * n_layers)(*budgets)
         self.cfg = OvggtConfig(n_layers, n_heads, head_dim, n_special, grid_h, grid_w, self._budgets,
                                anchor_tokens, k_max, min_anchor_interval, tau, alpha, beta,
-                               protect_first_frame, score_mode, dtype, compaction, None, 0)
+                               protect_first_frame, score_mode, dtype, compaction, camera_head, None, 0)
         self.compaction = compaction
         self.M = n_special + grid_h * grid_w
         self.C = n_heads * head_dim
@@ -224,6 +229,26 @@ class OvggtCache:
         io = self._io(frame_id, resid=resid, conf=conf, rho=rho, score_override=score_override)
         _check(lib().ovggt_layer_compress(self._h, layer, C.byref(io), _stream_ptr(stream)), "ovggt_layer_compress")
 
+    def anchor_decision(self, frame_id):
+        """(registered, demoted_frame) of frame_id as this (aggregator) handle decided it."""
+        reg, dem = C.c_int32(0), C.c_int64(-1)
+        _check(lib().ovggt_cache_anchor_decision(self._h, int(frame_id), C.byref(reg), C.byref(dem)),
+               "ovggt_cache_anchor_decision")
+        return bool(reg.value), int(dem.value)
+
+    def camera_compress(self, layer, frame_id, resid, registered, demoted_frame, score_override=None, stream=None) -> None:
+        io = self._io(frame_id, resid=resid, score_override=score_override)
+        _check(lib().ovggt_camera_compress(self._h, layer, C.byref(io), int(bool(registered)), int(demoted_frame),
+                                           _stream_ptr(stream)), "ovggt_camera_compress")
+
+    @classmethod
+    def camera(cls, *, n_layers=1, n_heads=16, head_dim=64, budget=144, k_max=3, beta=0.5, protect_first_frame=1,
+               score_mode=SCORE_HYBRID, dtype=DTYPE_BF16, **kw) -> "OvggtCache":
+        """The camera head's cache (Supp. C): one token per frame."""
+        return cls(n_layers=n_layers, n_heads=n_heads, head_dim=head_dim, n_special=1, grid_h=0, grid_w=0,
+                   budget=budget, anchor_tokens=0, k_max=k_max, beta=beta, protect_first_frame=protect_first_frame,
+                   score_mode=score_mode, dtype=dtype, camera_head=1, **kw)
+
     def layer_step(self, layer, frame_id, q, k, v, resid, conf=None, rho=float("nan"), score_override=None,
                    out=None, stream=None) -> torch.Tensor:
         out = self.new_out() if out is None else out
@@ -263,6 +288,17 @@ class OvggtCache:
         _check(lib().ovggt_cache_import(self._h, layer, ids.ctypes.data, flags.ctypes.data, scores.ctypes.data,
                                         k.ctypes.data, v.ctypes.data, len(ids), int(next_frame_id),
                                         int(last_registration_frame)), "ovggt_cache_import")
+
+    def selftest_bounded_wait(self, limit_us: int, stream=None) -> int:
+        """Runs the library's bounded device-side wait on a barrier nothing completes; returns the nanoseconds it
+        waited.  The handle's status word then holds the time-out code until clear_status()."""
+        ns = C.c_uint64(0)
+        _check(lib().ovggt_cache_selftest_bounded_wait(self._h, int(limit_us), C.byref(ns), _stream_ptr(stream)),
+               "ovggt_cache_selftest_bounded_wait")
+        return int(ns.value)
+
+    def clear_status(self) -> None:
+        _check(lib().ovggt_cache_clear_status(self._h), "ovggt_cache_clear_status")
 
     def reset(self) -> None:
         _check(lib().ovggt_cache_reset(self._h), "ovggt_cache_reset")

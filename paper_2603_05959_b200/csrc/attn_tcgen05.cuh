@@ -22,6 +22,7 @@
 
 #include <cuda.h>
 
+#include <algorithm>
 #include <type_traits>
 
 #include "common.cuh"
@@ -85,8 +86,12 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
-// Wait for the phase with the given parity, for at most about one second.
-__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, AttnBarriers* B, int* status) {
+// Wait for the phase with the given parity, for at most limit_ns (about one second unless stated).  On expiry the
+// CTA's abort flag is raised, OVGGT_ERR_TIMEOUT goes to the status word and the caller gets false; so does every
+// other waiter of the CTA the next time it looks at the flag.
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;
+__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, AttnBarriers* B, int* status,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   unsigned long long t0 = 0;
   for (uint32_t spins = 1;; ++spins) {
@@ -95,7 +100,7 @@ __device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, AttnBarrie
       if (*(volatile int*)&B->abort_flag) return false;
       const unsigned long long now = global_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > 1000000000ull) {
+      else if (now - t0 > limit_ns) {
         *(volatile int*)&B->abort_flag = 1;
         atomicCAS(status, 0, OVGGT_ERR_TIMEOUT);
         return false;
@@ -447,7 +452,8 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     bool ok = true;
     for (int idx = 0; idx < 2 * n_tiles; ++idx) {       // idx = 2 * tile + half
       const int it = idx >> 1, hf = idx & 1;
-      ok = mbar_wait(&B->s_full[hf], (uint32_t)it & 1u, B, P.status);
+      // (every wait result is made warp-uniform before the warp meets an .aligned tensor-memory instruction)
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(&B->s_full[hf], (uint32_t)it & 1u, B, P.status)) != 0;
       if (!ok) break;
       tc_fence_after();
       uint32_t s[kHalf];
@@ -514,6 +520,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           // idx + 1, so the completion of those scores covers it; the last half has a barrier of its own.
           ok = idx + 1 < 2 * n_tiles ? mbar_wait(&B->s_full[hf ^ 1], (uint32_t)((idx + 1) >> 1) & 1u, B, P.status)
                                      : mbar_wait(&B->pv_done, 0, B, P.status);
+          ok = __all_sync(0xFFFFFFFFu, ok) != 0;
           if (!ok) break;
           tc_fence_after();
           const float a = grow ? ex2(mref - mx) : 1.0f;
@@ -543,6 +550,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_arrive(&B->p_full[hf]);
     }
     if (ok) ok = mbar_wait(&B->o_full, 0, B, P.status);
+    ok = __all_sync(0xFFFFFFFFu, ok) != 0;
     if (ok) {
       tc_fence_after();
       const int m = qt * kBM + row;
@@ -625,6 +633,24 @@ __global__ void __launch_bounds__(256) k_attn_merge(const float* __restrict__ o_
   w.x = pack_bf16(acc.x * inv, acc.y * inv);
   w.y = pack_bf16(acc.z * inv, acc.w * inv);
   *reinterpret_cast<uint2*>(out + (size_t)m * C + c4 * 4) = w;
+}
+
+// Self-test of the bounded wait: one CTA sets up a barrier that expects one arrival, nobody arrives, and the wait is
+// given limit_ns.  The kernel must come back with OVGGT_ERR_TIMEOUT in the status word (no tensor memory, no bulk
+// copy, nothing in flight when it returns).  waited_ns receives how long the wait lasted.
+__global__ void __launch_bounds__(32) k_bounded_wait_selftest(int* status, unsigned long long limit_ns,
+                                                              unsigned long long* waited_ns) {
+  __shared__ AttnBarriers B;
+  if (threadIdx.x == 0) {
+    mbar_init(&B.q_full, 1);
+    B.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  const unsigned long long t0 = global_ns();
+  const bool ok = __all_sync(0xFFFFFFFFu, mbar_wait(&B.q_full, 0, &B, status, limit_ns)) != 0;
+  if (threadIdx.x == 0 && waited_ns) *waited_ns = global_ns() - t0;
+  if (ok && threadIdx.x == 0) atomicCAS(status, 0, OVGGT_ERR_DEVICE_STATUS);   // a wait nobody ends must not succeed
 }
 
 // ---------------------------------------------------------------- host side
@@ -715,7 +741,8 @@ inline int attn_kv_maps(AttnKvMaps* m, const void* k, const void* v, int N, int 
 }
 
 inline int attn_tcgen05_launch(const void* q, const void* k, const void* v, int M, int N, int H, void* out,
-                               void* scratch, int* status, cudaStream_t st, AttnKvMaps* kv_maps = nullptr) {
+                               void* scratch, int* status, cudaStream_t st, AttnKvMaps* kv_maps = nullptr,
+                               int force_splits = 0) {
   const int C = H * kHD;
   CUtensorMap tq;
   AttnKvMaps local;
@@ -729,8 +756,9 @@ inline int attn_tcgen05_launch(const void* q, const void* k, const void* v, int 
   AttnParams P;
   P.M = M; P.N = N; P.H = H;
   P.tiles_total = (N + kBN - 1) / kBN;
-  P.splits = attn_choose_splits(M, N, H);
+  P.splits = force_splits > 0 ? std::min(force_splits, std::min(kMaxSplits, P.tiles_total)) : attn_choose_splits(M, N, H);
   P.tiles_per_split = (P.tiles_total + P.splits - 1) / P.splits;
+  P.splits = (P.tiles_total + P.tiles_per_split - 1) / P.tiles_per_split;     // no empty split
   P.out = static_cast<__nv_bfloat16*>(out);
   P.o_part = static_cast<float*>(scratch);
   P.ml_part = reinterpret_cast<float2*>(static_cast<char*>(scratch) + (size_t)kMaxSplits * M * C * 4);

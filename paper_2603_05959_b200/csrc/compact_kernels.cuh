@@ -154,17 +154,28 @@ constexpr int kFillSlices = 16;
 constexpr int kFillClusterCtas = 8;
 constexpr int kFillThreads = 256;
 
+struct FillArgs {
+  uint4* k_cache; uint4* v_cache;
+  const int* move_src; const int* move_dst; const int* move_j; const int* n_moves_ptr;
+  int max_moves;
+  int* slot_meta;
+  float* delta;                 // [kFillSlices, C] or nullptr
+};
+
 template <int DT>
-__global__ void __launch_bounds__(kFillThreads) k_fill_holes(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
-                                                             const int* __restrict__ move_src,
-                                                             const int* __restrict__ move_dst,
-                                                             const int* __restrict__ move_j,
-                                                             const int* __restrict__ n_moves_ptr, int max_moves,
-                                                             int nvec, int* __restrict__ slot_meta,
-                                                             float* __restrict__ delta /* [kFillSlices, C] or null */) {
+__device__ __forceinline__ void fill_holes_body(const FillArgs& A, int nvec) {
   constexpr int VEC = VecOf<DT>::n;
   __shared__ __align__(16) float red[4][kCompactSumMaxVec * VEC];
   __shared__ __align__(16) float cta_part[kCompactSumMaxVec * VEC];
+  uint4* __restrict__ k_cache = A.k_cache;
+  uint4* __restrict__ v_cache = A.v_cache;
+  const int* __restrict__ move_src = A.move_src;
+  const int* __restrict__ move_dst = A.move_dst;
+  const int* __restrict__ move_j = A.move_j;
+  const int* __restrict__ n_moves_ptr = A.n_moves_ptr;
+  int* __restrict__ slot_meta = A.slot_meta;
+  float* __restrict__ delta = A.delta;
+  const int max_moves = A.max_moves;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
   const int n_moves = min(*n_moves_ptr, max_moves);
@@ -236,6 +247,29 @@ __global__ void __launch_bounds__(kFillThreads) k_fill_holes(uint4* __restrict__
     delta[(size_t)cid * C + c] = t;
   }
   cluster.sync();   // no CTA may exit while others still read its shared memory
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kFillThreads) k_fill_holes(uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
+                                                             const int* __restrict__ move_src,
+                                                             const int* __restrict__ move_dst,
+                                                             const int* __restrict__ move_j,
+                                                             const int* __restrict__ n_moves_ptr, int max_moves,
+                                                             int nvec, int* __restrict__ slot_meta,
+                                                             float* __restrict__ delta /* [kFillSlices, C] or null */) {
+  const FillArgs A{k_cache, v_cache, move_src, move_dst, move_j, n_moves_ptr, max_moves, slot_meta, delta};
+  fill_holes_body<DT>(A, nvec);
+}
+
+// The moves of several layers in one launch: blockIdx.y = position in the batch.  (A layer of the batch without
+// corrections to compute returns before the cluster barriers; all CTAs of its clusters do, so nobody is left waiting.)
+constexpr int kMaxFillBatch = 32;
+struct FillBatch {
+  FillArgs a[kMaxFillBatch];
+};
+template <int DT>
+__global__ void __launch_bounds__(kFillThreads) k_fill_holes_batched(const __grid_constant__ FillBatch batch, int nvec) {
+  fill_holes_body<DT>(batch.a[blockIdx.y], nvec);
 }
 
 }  // namespace ovggt

@@ -354,7 +354,12 @@ bool config_ok(const ovggt_config* c, int* err) {
   *err = OVGGT_ERR_INVALID_ARG;
   if (!c || !c->budget) return false;
   if (c->n_layers < 1 || c->n_heads < 1 || c->head_dim != 64) return false;
-  if (c->n_special < 0 || c->grid_h < 1 || c->grid_w < 1) return false;
+  if (c->camera_head != 0 && c->camera_head != 1) return false;
+  if (c->camera_head) {   // Supp. C: one camera token per frame and nothing else
+    if (c->n_special != 1 || c->grid_h != 0 || c->grid_w != 0 || c->anchor_tokens != 0) return false;
+  } else if (c->n_special < 0 || c->grid_h < 1 || c->grid_w < 1) {
+    return false;
+  }
   if (c->anchor_tokens < 0 || c->anchor_tokens > c->grid_h * c->grid_w) return false;
   if (c->k_max < 0 || c->k_max > OVGGT_MAX_ANCHORS || c->min_anchor_interval < 0) return false;
   if (c->dtype != kF32 && c->dtype != kBF16) return false;
@@ -362,7 +367,8 @@ bool config_ok(const ovggt_config* c, int* err) {
   if (c->compaction != OVGGT_COMPACT_FILL_HOLES && c->compaction != OVGGT_COMPACT_STABLE_GATHER) return false;
   if (!(c->alpha >= 0.0f && c->alpha <= 1.0f) || !(c->beta >= 0.0f && c->beta <= 1.0f)) return false;
   const int64_t M = c->n_special + (int64_t)c->grid_h * c->grid_w;
-  const int64_t pmax = (c->protect_first_frame ? M : 0) + (int64_t)c->k_max * c->anchor_tokens;
+  // Eq. 9; in the camera head's cache an anchor is the frame's one token
+  const int64_t pmax = (c->protect_first_frame ? M : 0) + (int64_t)c->k_max * (c->camera_head ? 1 : c->anchor_tokens);
   for (int l = 0; l < c->n_layers; ++l) {
     if (c->budget[l] < M || c->budget[l] < pmax) {
       *err = OVGGT_ERR_BUDGET_TOO_SMALL;
@@ -672,10 +678,16 @@ int enqueue_scores(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io, cuda
 // writes another buffer and may run beside an attention that still reads this one (st_move = st_sel); the
 // hole-filling move writes the buffer the attention reads, so it follows both (st_move = the attention's stream,
 // which first waits for st_sel).
-int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st_sel, cudaStream_t st_move) {
+// `mirrored`: the anchor decision of the frame as another handle took it (camera head, Supp. C) instead of the rule
+// of Sec. 3.3 applied to rho.
+struct MirroredDecision { bool registered; int64_t demoted_frame; };
+
+int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st_sel, cudaStream_t st_move,
+                  const MirroredDecision* mirrored = nullptr) {
   int rc = check_layer(h, layer);
   if (rc) return rc;
   if (!io || !io->resid) return OVGGT_ERR_INVALID_ARG;
+  if ((h->cfg.camera_head != 0) != (mirrored != nullptr)) return OVGGT_ERR_INVALID_ARG;
   if (!aligned16(io->resid)) return OVGGT_ERR_MISALIGNED;
   LayerState& S = h->layers[layer];
   if (!S.pending || io->frame_id != S.pending_frame) return OVGGT_ERR_FRAME_ORDER;
@@ -696,8 +708,22 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
     h->decided_frame = t;
     h->decided_register = false;
     h->decided_demote = -1;
-    if (t != h->first_frame && c.anchor_tokens > 0 && c.k_max > 0 && io->conf != nullptr && io->rho < c.tau &&
-        t - h->last_registration >= c.min_anchor_interval) {
+    if (mirrored) {
+      // the frame's token is protected / the demoted frame's token released exactly when the aggregator did so
+      if (t != h->first_frame && mirrored->registered && (int)h->anchors.size() < OVGGT_MAX_ANCHORS) {
+        h->decided_register = true;
+        h->anchors.push_back(t);
+        h->last_registration = t;
+      }
+      if (mirrored->demoted_frame >= 0) {
+        auto it = std::find(h->anchors.begin(), h->anchors.end(), mirrored->demoted_frame);
+        if (it != h->anchors.end()) {
+          h->decided_demote = mirrored->demoted_frame;
+          h->anchors.erase(it);
+        }
+      }
+    } else if (t != h->first_frame && c.anchor_tokens > 0 && c.k_max > 0 && io->conf != nullptr && io->rho < c.tau &&
+               t - h->last_registration >= c.min_anchor_interval) {
       h->decided_register = true;
       h->anchors.push_back(t);
       h->last_registration = t;
@@ -707,6 +733,7 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
       }
     }
   }
+  const int per_anchor = c.camera_head ? 1 : c.anchor_tokens;
   const bool first = (t == h->first_frame);
   h->last_stream = st_move;
 
@@ -722,8 +749,10 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
   P.alpha = c.alpha; P.w_center = h->w_center; P.w_edge = h->w_edge; P.w_corner = h->w_corner;
   P.beta = c.beta;
   P.mode = c.score_mode;
-  P.protect_new = (first && c.protect_first_frame) ? 1 : 0;
-  P.register_anchor = h->decided_register ? 1 : 0;
+  P.protect_new = (first && c.protect_first_frame) ? OVGGT_FLAG_INIT
+                                                   : ((c.camera_head && h->decided_register) ? OVGGT_FLAG_HIST : 0);
+  P.lone_new = c.camera_head ? 1.0f : -1.0f;
+  P.register_anchor = (!c.camera_head && h->decided_register) ? 1 : 0;
   P.A = c.anchor_tokens;
   P.demote_frame = h->decided_demote;
   P.s_raw = S.s_raw; P.d = S.d; P.conf = io->conf; P.override_r = io->score_override;
@@ -776,8 +805,8 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
 
   // bookkeeping that follows deterministically from the sizes
   if (first && c.protect_first_frame) S.n_prot_init = M;
-  if (h->decided_register) S.n_prot_hist += c.anchor_tokens;
-  if (h->decided_demote >= 0) S.n_prot_hist -= c.anchor_tokens;
+  if (h->decided_register) S.n_prot_hist += per_anchor;
+  if (h->decided_demote >= 0) S.n_prot_hist -= per_anchor;
   S.evicted_total += N - n_keep;
   S.last_N = N;
   S.last_keep = n_keep;
@@ -801,9 +830,27 @@ extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_f
   return compress_impl(h, layer, io, st, st);
 }
 
+extern "C" int ovggt_cache_anchor_decision(ovggt_cache* h, int64_t frame_id, int32_t* registered,
+                                           int64_t* demoted_frame) {
+  if (!h || !registered || !demoted_frame) return OVGGT_ERR_INVALID_ARG;
+  if (h->decided_frame != frame_id) return OVGGT_ERR_FRAME_ORDER;
+  *registered = h->decided_register ? 1 : 0;
+  *demoted_frame = h->decided_demote;
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_camera_compress(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, int32_t registered,
+                                     int64_t demoted_frame, void* stream) {
+  if (!h || !h->cfg.camera_head) return OVGGT_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const MirroredDecision d{registered != 0, demoted_frame};
+  return compress_impl(h, layer, io, st, st, &d);
+}
+
 extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
   int rc = check_layer(h, layer);
   if (rc) return rc;
+  if (h->cfg.camera_head) return OVGGT_ERR_INVALID_ARG;   // the camera head's cache needs the aggregator's decision
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const bool can_overlap = h->side && h->overlap && io && io->resid && aligned16(io->resid) && io->q && io->k &&
                            io->v && io->out && !h->layers[layer].pending;
@@ -1056,6 +1103,29 @@ extern "C" int ovggt_cache_reset(ovggt_cache* h) {
   h->decided_register = false;
   h->decided_demote = -1;
   CK(cudaMemset(h->status, 0, 64));
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_cache_clear_status(ovggt_cache* h) {
+  if (!h) return OVGGT_ERR_INVALID_ARG;
+  CK(cudaStreamSynchronize(h->last_stream));
+  CK(cudaMemset(h->status, 0, 64));
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_cache_selftest_bounded_wait(ovggt_cache* h, uint32_t limit_us, uint64_t* waited_ns, void* stream) {
+  if (!h || limit_us == 0 || limit_us > 1000000) return OVGGT_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  h->last_stream = st;
+  unsigned long long* dev_ns = reinterpret_cast<unsigned long long*>(h->status + 8);   // (inside the 64-byte status block)
+  k_bounded_wait_selftest<<<1, 32, 0, st>>>(h->status, (unsigned long long)limit_us * 1000ull, dev_ns);
+  LAUNCHED();
+  if (waited_ns) {
+    CK(cudaStreamSynchronize(st));
+    unsigned long long ns = 0;
+    CK(cudaMemcpy(&ns, dev_ns, 8, cudaMemcpyDeviceToHost));
+    *waited_ns = ns;
+  }
   return OVGGT_OK;
 }
 

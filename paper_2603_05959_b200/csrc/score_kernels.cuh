@@ -141,22 +141,31 @@ __global__ void __launch_bounds__(1024) k_colsum_final_sliced(const float* __res
 // sums themselves; more: a base row plus corrections, as the hole-filling compaction leaves them).  A zero vector has cosine 0.  One warp per pair of rows; ksum is staged in shared memory
 // once per CTA and, for rows of up to 128 vectors, kept in registers by the lanes that meet its columns;
 // |ksum|^2 is folded by every warp in the same order, so all CTAs agree on it.
+struct DiversityArgs {
+  const uint4* K; int rows;                 // cached keys [rows, C]
+  const float* ksum; int n_slices;          // [n_slices, C]
+  float* ksum_out;                          // [C] or nullptr
+  float* d;                                 // [rows]
+  int div_ctas;                             // CTAs [0, div_ctas) of the launch work on d; later ones on the norms
+  const uint4* resid; int resid_rows;       // [resid_rows, C] or nullptr
+  float* s_raw;                             // [resid_rows]
+};
+
 template <int DT>
-__global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, int rows, int nvec,
-                                                   const float* __restrict__ ksum, int n_slices,
-                                                   float* __restrict__ ksum_out,
-                                                   float* __restrict__ d, int div_ctas,
-                                                   const uint4* __restrict__ resid, int resid_rows,
-                                                   float* __restrict__ s_raw) {
+__device__ __forceinline__ void diversity_body(const DiversityArgs& A, int nvec, float* sh_ksum) {
   constexpr int VEC = VecOf<DT>::n;
+  const uint4* __restrict__ K = A.K;
+  const float* __restrict__ ksum = A.ksum;
+  float* __restrict__ ksum_out = A.ksum_out;
+  float* __restrict__ d = A.d;
+  const int rows = A.rows, n_slices = A.n_slices, div_ctas = A.div_ctas;
   // CTAs past the first div_ctas carry a second, independent job in the same launch: the residual norms of
   // Eq. 5 (one warp per row), so that a step pays one launch for both scores.
   if ((int)blockIdx.x >= div_ctas) {
     const int row = (int)((((int)blockIdx.x - div_ctas) * (unsigned)blockDim.x + threadIdx.x) >> 5);
-    if (row < resid_rows) warp_row_norm<DT>(resid, row, nvec, s_raw);
+    if (A.resid != nullptr && row < A.resid_rows) warp_row_norm<DT>(A.resid, row, nvec, A.s_raw);
     return;
   }
-  extern __shared__ __align__(16) float sh_ksum[];
   const int C = nvec * VEC;
   const int lane = threadIdx.x & 31;
   const int warps_total = (int)((div_ctas * (unsigned)blockDim.x) >> 5);
@@ -248,6 +257,30 @@ __global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, 
       }
     }
   }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(256) k_diversity(const uint4* __restrict__ K, int rows, int nvec,
+                                                   const float* __restrict__ ksum, int n_slices,
+                                                   float* __restrict__ ksum_out,
+                                                   float* __restrict__ d, int div_ctas,
+                                                   const uint4* __restrict__ resid, int resid_rows,
+                                                   float* __restrict__ s_raw) {
+  extern __shared__ __align__(16) float sh_ksum[];
+  const DiversityArgs A{K, rows, ksum, n_slices, ksum_out, d, div_ctas, resid, resid_rows, s_raw};
+  diversity_body<DT>(A, nvec, sh_ksum);
+}
+
+// Both scores of several layers in one launch: blockIdx.y = position in the batch, every layer with its own cache,
+// sums and residual; the grid's x extent is the largest layer's, smaller layers leave their surplus CTAs idle.
+constexpr int kMaxScoreBatch = 32;
+struct DiversityBatch {
+  DiversityArgs a[kMaxScoreBatch];
+};
+template <int DT>
+__global__ void __launch_bounds__(256) k_diversity_batched(const __grid_constant__ DiversityBatch batch, int nvec) {
+  extern __shared__ __align__(16) float sh_ksum[];
+  diversity_body<DT>(batch.a[blockIdx.y], nvec, sh_ksum);
 }
 
 }  // namespace ovggt

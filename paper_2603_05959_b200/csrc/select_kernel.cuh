@@ -277,7 +277,8 @@ struct CompressParams {
   float alpha, w_center, w_edge, w_corner;   // Eq. 6: blend and the normalised 3x3 Gaussian weights
   float beta;
   int mode;                         // OVGGT_SCORE_*
-  int protect_new;                  // 1: flag the new rows INIT (first frame)
+  int protect_new;                  // != 0: give every new row this flag (INIT: first frame; HIST: a camera-cache anchor)
+  float lone_new;                   // >= 0: normalised score of a new group without a range (Eq. 7's 0/0); < 0: 0
   int register_anchor, A;           // 1: flag the A most confident patches of the new frame HIST
   long long demote_frame;           // >= 0: release the HIST rows of that frame
   const float* s_raw;               // [M] residual norms of the new rows
@@ -322,8 +323,7 @@ __device__ __forceinline__ float smoothed_score(const CompressParams& P, const f
   return v;
 }
 
-__global__ void __launch_bounds__(kSelectThreads) k_compress_select(const CompressParams P) {
-  extern __shared__ __align__(16) unsigned char smem[];
+__device__ __forceinline__ void compress_select_body(const CompressParams& P, unsigned char* smem) {
   cg::cluster_group cluster = cg::this_cluster();
   const int ncta = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   SelectShared* sh = reinterpret_cast<SelectShared*>(smem);
@@ -393,7 +393,7 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
         float x, keepscore;
         if (g >= n) {
           const int j = g - n;
-          if (P.protect_new) f = OVGGT_FLAG_INIT;
+          if (P.protect_new) f = (uint8_t)P.protect_new;
           if (reg && j >= P.n_special && cmark[j - P.n_special]) f = OVGGT_FLAG_HIST;
           x = smoothed_score(P, sraw, j);
           keepscore = x;           // the score the row keeps
@@ -456,7 +456,8 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
       if (P.mode == OVGGT_SCORE_HYBRID) {
         const float lo = g < n ? lo_h : lo_n, hi = g < n ? hi_h : hi_n;
         const float w = g < n ? 1.0f - P.beta : P.beta;
-        r = hi > lo ? __fmul_rn(w, __fdiv_rn(val[i] - lo, hi - lo)) : 0.0f;
+        r = hi > lo ? __fmul_rn(w, __fdiv_rn(val[i] - lo, hi - lo))
+                    : ((g >= n && P.lone_new >= 0.0f) ? __fmul_rn(w, P.lone_new) : 0.0f);
       } else {
         r = val[i];
       }
@@ -546,6 +547,22 @@ __global__ void __launch_bounds__(kSelectThreads) k_compress_select(const Compre
     }
   }
   cluster.sync();   // no CTA may exit while others still read its shared memory
+}
+
+__global__ void __launch_bounds__(kSelectThreads) k_compress_select(const CompressParams P) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  compress_select_body(P, smem);
+}
+
+// The same step for several layers in one launch (Sec. 3.2: every layer has its own budget B^(l) and cache): one
+// cluster per layer, blockIdx.y = position in the batch.  The parameter blocks travel as kernel arguments.
+constexpr int kMaxBatchLayers = 32;
+struct CompressBatch {
+  CompressParams p[kMaxBatchLayers];
+};
+__global__ void __launch_bounds__(kSelectThreads) k_compress_select_batched(const __grid_constant__ CompressBatch batch) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  compress_select_body(batch.p[blockIdx.y], smem);
 }
 
 }  // namespace ovggt

@@ -115,7 +115,9 @@ def _randn(shape, std, device, dtype, gen_):
 class ProjectionStack:
     """24 global-attention layers with their own caches.  Per layer: q, k, v = x W_qkv (random-init N(0, 0.02)),
     the library attends, x <- x + O W_o.  There is no MLP in this workload, so the residual that feeds the activation
-    score is the seeded synthetic one of the single-layer workload.  `tap`, if given, receives every library input."""
+    score is the seeded synthetic one of the single-layer workload.  `tap(t, l, q, k, v, resid)`, if given, sees every
+    library input and may return priorities to rank instead of the library's own (teacher forcing in the tests);
+    `after(t, l, out)` sees the attention output of every library call."""
 
     def __init__(self, cfg: gen.StreamConfig, device, compaction: int = B.COMPACT_FILL_HOLES):
         assert cfg.dtype == gen.DTYPE_BF16
@@ -128,6 +130,7 @@ class ProjectionStack:
         self.w_o = [_randn((C, C), 0.02, device, torch.bfloat16, g) for _ in range(L)]
         self.out = self.cache.new_out()
         self.tap: Optional[Callable] = None
+        self.after: Optional[Callable] = None
 
     def frame(self, t: int, x: torch.Tensor, resid: List[torch.Tensor], conf: torch.Tensor, rho: float, stream,
               lib: Optional[_Timer] = None) -> torch.Tensor:
@@ -137,10 +140,12 @@ class ProjectionStack:
             # embeddings are N(0, 1) over 1024 columns and the weights N(0, 0.02): q, k, v come out near N(0, 0.4)
             qkv = x @ self.w_qkv[l]
             q, k, v = (qkv[:, i * C:(i + 1) * C].contiguous() for i in range(3))
-            if self.tap:
-                self.tap(t, l, q, k, v, resid[l])
-            run = lambda: self.cache.layer_step(l, t, q, k, v, resid[l], conf, rho, out=self.out, stream=stream)
+            ov = self.tap(t, l, q, k, v, resid[l]) if self.tap else None
+            run = lambda: self.cache.layer_step(l, t, q, k, v, resid[l], conf, rho, score_override=ov, out=self.out,
+                                                stream=stream)
             lib(run) if lib else run()
+            if self.after:
+                self.after(t, l, self.out)
             x = x + self.out @ self.w_o[l]
         return x
 
@@ -157,7 +162,7 @@ class Aggregator:
     global-attention block (the library: attention over the bounded cache), each followed by an MLP of width 4C,
     random-init N(0, 0.02), LayerScale taken as 1.  In the global block the library's two halves bracket the MLP:
     attend -> h = x + O W_o -> r = MLP(LN(h)) -> compress(resid = r) -> x = h + r, so the activation score sees the
-    block's real MLP output.  `tap`, if given, receives every library input."""
+    block's real MLP output.  `tap` and `after` as in ProjectionStack."""
 
     def __init__(self, cfg: gen.StreamConfig, device, compaction: int = B.COMPACT_FILL_HOLES):
         assert cfg.dtype == gen.DTYPE_BF16
@@ -171,6 +176,7 @@ class Aggregator:
                         for kind in ("frame", "global")} for _ in range(L)]
         self.out = self.cache.new_out()
         self.tap: Optional[Callable] = None
+        self.after: Optional[Callable] = None
 
     def _mlp(self, w, h):
         return torch.nn.functional.gelu(_layer_norm(h) @ w["fc1"]) @ w["fc2"]
@@ -190,11 +196,12 @@ class Aggregator:
             q, k, v = (qkv[:, i * C:(i + 1) * C].contiguous() for i in range(3))
             att = lambda: self.cache.layer_attend(l, t, q, k, v, out=self.out, stream=stream)
             lib(att) if lib else att()
+            if self.after:
+                self.after(t, l, self.out)
             h = x + self.out @ w["o"]
             r = self._mlp(w, h).contiguous()
-            if self.tap:
-                self.tap(t, l, q, k, v, r)
-            cmp_ = lambda: self.cache.layer_compress(l, t, r, conf, rho, stream=stream)
+            ov = self.tap(t, l, q, k, v, r) if self.tap else None
+            cmp_ = lambda: self.cache.layer_compress(l, t, r, conf, rho, score_override=ov, stream=stream)
             lib(cmp_) if lib else cmp_()
             x = h + r
         return x

@@ -82,6 +82,93 @@ def test_stack_of_24_layers_each_with_its_own_cache():
     assert all(x.evicted_total > 0 for x in o.values())
 
 
+def _follow_harness(model, cfg, n_frames, conf_rho, run_frame, rows):
+    """Teacher-forced check of the library calls a workload harness makes: the oracle of every layer is fed the
+    tensors the harness hands to the library (tap), its priorities are ranked on both sides, and the attention output
+    (after) and the survivors are compared call by call."""
+    orc.set_threads(16)
+    oracles = [orc.OracleLayer.from_stream(cfg) for _ in range(cfg.n_layers)]
+    pending, checked = {}, {"attn": 0, "sel": 0}
+
+    def tap(t, l, q, k, v, resid):
+        conf, rho = conf_rho(t)
+        f32 = lambda x: x.float().cpu().numpy()
+        ref_out = oracles[l].attend(t, f32(q), f32(k), f32(v), rows=rows)
+        ref = oracles[l].compress(f32(resid), conf, rho)
+        pending[(t, l)] = (ref_out, ref)
+        return torch.from_numpy(ref["r"]).cuda()
+
+    def after(t, l, out):
+        pending[("out", t, l)] = out_to_f32(out)[rows]
+
+    model.tap, model.after = tap, after
+    for t in range(n_frames):
+        run_frame(t)
+        for l in range(cfg.n_layers):
+            ref_out, ref = pending.pop((t, l))
+            got = pending.pop(("out", t, l))
+            err = np.abs(got - ref_out)
+            assert err.max() <= ATT_MAX and err.mean() <= ATT_MEAN, (t, l, err.max(), err.mean())
+            sel = model.cache.last_selection(l)
+            np.testing.assert_array_equal(sel["survivors"], ref["survivors"], err_msg=f"frame {t} layer {l}")
+            fin = np.isfinite(ref["r"])
+            np.testing.assert_allclose(sel["r"][fin], ref["r"][fin], rtol=0, atol=R_ATOL, err_msg=f"frame {t} layer {l}")
+            checked["attn"] += 1
+            checked["sel"] += 1
+            assert model.cache.stats(l)["device_status"] == 0
+    for l, o in enumerate(oracles):
+        ex, rx = model.cache.export(l), o.export()
+        np.testing.assert_array_equal(ex["ids"], rx["ids"])
+        np.testing.assert_array_equal(ex["flags"], rx["flags"])
+        assert np.array_equal(storage_to_f32(ex["k"], cfg.dtype), rx["k"])
+    return oracles, checked
+
+
+def test_projection_stack_harness_library_calls_match_the_oracle():
+    """The harness of the 24-layer workload (random-init QKV / output projections in torch around the library), cut
+    to 3 layers and a budget that the frames overflow: every library call against the oracle."""
+    from paper_2603_05959_b200 import harness as H
+    cfg = gen.config_stack24().replace(n_layers=3, budget=3000, min_anchor_interval=2, tau=0.8)
+    model = H.ProjectionStack(cfg, torch.device("cuda", torch.cuda.current_device()))
+    stream = torch.cuda.current_stream()
+    rows = np.array([0, 4, 5, 700, 1373], dtype=np.int32)
+
+    def conf_rho(t):
+        fi = gen.frame_inputs(cfg, t, fields=("anchor inputs only",))
+        return fi.conf, fi.rho
+
+    def run_frame(t):
+        conf, rho, resid = H.frame_side_inputs(cfg, t, model.device, cfg.n_layers)
+        model.frame(t, H.patch_embeddings(cfg, t, model.device), resid, conf, rho, stream)
+
+    oracles, checked = _follow_harness(model, cfg, 5, conf_rho, run_frame, rows)
+    assert checked["sel"] == 15 and all(o.evicted_total > 0 for o in oracles)
+    model.destroy()
+
+
+def test_aggregator_harness_library_calls_match_the_oracle():
+    """The alternating-aggregator harness (frame attention and MLPs in torch; attend -> MLP -> compress around the
+    library, the activation score fed by the block's real MLP output), cut to 2 depths: every library call against
+    the oracle, on the 1041-token layout."""
+    from paper_2603_05959_b200 import harness as H
+    cfg = gen.config_aggregator().replace(n_layers=2, budget=2500, min_anchor_interval=2, tau=0.8)
+    model = H.Aggregator(cfg, torch.device("cuda", torch.cuda.current_device()))
+    stream = torch.cuda.current_stream()
+    rows = np.array([0, 3, 5, 512, 1040], dtype=np.int32)
+
+    def conf_rho(t):
+        fi = gen.frame_inputs(cfg, t, fields=("anchor inputs only",))
+        return fi.conf, fi.rho
+
+    def run_frame(t):
+        conf, rho, _ = H.frame_side_inputs(cfg, t, model.device, 0)
+        model.frame(t, H.patch_embeddings(cfg, t, model.device), conf, rho, stream)
+
+    oracles, checked = _follow_harness(model, cfg, 5, conf_rho, run_frame, rows)
+    assert checked["sel"] == 10 and all(o.evicted_total > 0 for o in oracles)
+    model.destroy()
+
+
 @pytest.mark.parametrize("budget,anchors,mode,frames", [
     (4096, 0, gen.SCORE_HYBRID, 12),
     (4096, 256, gen.SCORE_RESIDUAL_STORED, 12),

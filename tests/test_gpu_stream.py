@@ -255,6 +255,38 @@ def test_layers_must_compress_frames_in_order_across_the_handle():
     c.destroy()
 
 
+def test_bounded_device_wait_runs_out_cleanly_and_the_handle_recovers():
+    """Failure detection without a fault: the wait routine of the attention kernel is run on a barrier that nothing
+    completes, with a 2 ms limit.  The kernel returns, the status word and ovggt_cache_stats report the time-out,
+    the context stays usable, and after clearing the status the same handle passes a teacher-forced step."""
+    cfg = gen.config_tiny()
+    c = B.OvggtCache.from_stream(cfg)
+    layer = orc.OracleLayer.from_stream(cfg)
+
+    def forced_step(t):
+        fi = gen.frame_inputs(cfg, t)
+        df = DeviceFrame(cfg, fi, "cuda")
+        ref_out = layer.attend(t, fi.q, fi.k, fi.v)
+        ref = layer.compress(fi.resid, fi.conf, fi.rho)
+        out = c.layer_step(0, t, df.q, df.k, df.v, df.resid, df.conf, df.rho, score_override=torch.from_numpy(ref["r"]).cuda())
+        assert np.abs(out_to_f32(out) - ref_out).max() <= ATT_F32
+        np.testing.assert_array_equal(c.last_selection(0)["survivors"], ref["survivors"])
+
+    forced_step(0)
+    assert c.stats(0)["device_status"] == 0
+    waited = c.selftest_bounded_wait(2000)
+    assert 2_000_000 <= waited < 200_000_000                 # gave up after the limit, long before the default second
+    with pytest.raises(B.OvggtError) as e:
+        c.stats(0)
+    assert e.value.code == -9                                  # OVGGT_ERR_TIMEOUT, surfaced by the next stats call
+    torch.cuda.synchronize()                                   # the context is intact
+    c.clear_status()
+    for t in range(1, 6):
+        forced_step(t)
+    assert c.stats(0)["device_status"] == 0
+    c.destroy()
+
+
 def test_call_order_errors():
     cfg = gen.config_tiny()
     c = B.OvggtCache.from_stream(cfg)
