@@ -21,7 +21,7 @@ class OrcConfig(C.Structure):
         ("k_max", C.c_int32), ("min_anchor_interval", C.c_int32),
         ("tau", C.c_double), ("alpha", C.c_double), ("beta", C.c_double),
         ("protect_first_frame", C.c_int32), ("score_mode", C.c_int32),
-        ("diversity_per_head", C.c_int32), ("camera_cache", C.c_int32),
+        ("diversity_per_head", C.c_int32), ("camera_cache", C.c_int32), ("random_seed", C.c_uint64),
     ]
 
 
@@ -74,6 +74,10 @@ def lib():
         L.orc_full_cache_elements.restype = C.c_double
         L.orc_full_cache_elements.argtypes = [C.c_int32, C.c_int64, C.c_int32, C.c_int32, C.c_int32]
         L.orc_set_threads.argtypes = [C.c_int32]
+        L.orc_splitmix64.restype = C.c_uint64
+        L.orc_splitmix64.argtypes = [C.c_uint64]
+        L.orc_random_priority.restype = C.c_float
+        L.orc_random_priority.argtypes = [C.c_uint64, C.c_int64, C.c_int64]
         _LIB = L
     return _LIB
 
@@ -154,6 +158,14 @@ def attention(Q, K, V, n_heads: int, head_dim: int, rows: Optional[Sequence[int]
     return out
 
 
+def splitmix64(x: int) -> int:
+    return int(lib().orc_splitmix64(C.c_uint64(x & (2 ** 64 - 1))))
+
+
+def random_priority(seed: int, frame_id: int, token_id: int) -> float:
+    return float(lib().orc_random_priority(C.c_uint64(seed & (2 ** 64 - 1)), int(frame_id), int(token_id)))
+
+
 def full_cache_elements(L: int, T: int, M: int, n_heads: int, head_dim: int) -> float:
     return float(lib().orc_full_cache_elements(L, T, M, n_heads, head_dim))
 
@@ -165,10 +177,10 @@ class OracleLayer:
 
     def __init__(self, *, n_heads, head_dim, n_special, grid_h, grid_w, budget, anchor_tokens,
                  k_max=3, min_anchor_interval=100, tau=0.2, alpha=0.5, beta=0.5,
-                 protect_first_frame=1, score_mode=0, diversity_per_head=0, camera_cache=0):
+                 protect_first_frame=1, score_mode=0, diversity_per_head=0, camera_cache=0, random_seed=0):
         self.cfg = OrcConfig(n_heads, head_dim, n_special, grid_h, grid_w, budget, anchor_tokens,
                              k_max, min_anchor_interval, tau, alpha, beta, protect_first_frame,
-                             score_mode, diversity_per_head, camera_cache)
+                             score_mode, diversity_per_head, camera_cache, random_seed)
         self.M = n_special + grid_h * grid_w
         self.C = n_heads * head_dim
         self._h = lib().orc_create(C.byref(self.cfg))
@@ -182,7 +194,7 @@ class OracleLayer:
                   anchor_tokens=cfg.anchor_tokens, k_max=cfg.k_max,
                   min_anchor_interval=cfg.min_anchor_interval, tau=cfg.tau, alpha=cfg.alpha,
                   beta=cfg.beta, protect_first_frame=cfg.protect_first_frame,
-                  score_mode=cfg.score_mode)
+                  score_mode=cfg.score_mode, random_seed=cfg.seed)
         kw.update(over)
         return cls(**kw)
 

@@ -121,6 +121,20 @@ extern "C" void orc_hybrid(const double* d, const double* s, const uint8_t* flag
   minmax_group(s, flags + n, M, beta, r + n);
 }
 
+/* ------------------------------------------------------------------ random-eviction baseline (Supp. A) */
+extern "C" uint64_t orc_splitmix64(uint64_t x) {
+  uint64_t z = x + 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+extern "C" float orc_random_priority(uint64_t seed, int64_t frame_id, int64_t token_id) {
+  const uint64_t step_key = orc_splitmix64(seed ^ (uint64_t)frame_id);
+  const uint64_t bits = orc_splitmix64(step_key + (uint64_t)token_id);
+  return (float)(bits >> 40) * (1.0f / 16777216.0f); /* 24 bits: exact in fp32, in [0, 1) */
+}
+
 /* ------------------------------------------------------------------ Eq. 8 */
 /* Rank of a priority: NaN ranks with -inf (evicted first); -0 and +0 compare equal. */
 static inline float rank_key(float x) {
@@ -357,6 +371,10 @@ extern "C" int orc_compress(orc_state* st, const float* resid, const float* conf
     std::vector<double> d(std::max(n, 1));
     orc_diversity(st->k.data(), n, C, cfg.n_heads, cfg.diversity_per_head, d.data());
     orc_hybrid(d.data(), s_smooth.data(), st->flags.data(), n, M, cfg.beta, r.data());
+  } else if (cfg.score_mode == ORC_SCORE_RANDOM) {
+    for (int32_t i = 0; i < N; ++i)
+      r[i] = st->flags[i] != ORC_FLAG_EVICTABLE ? std::numeric_limits<float>::infinity()
+                                                : orc_random_priority(cfg.random_seed, t, st->ids[i]);
   } else {
     for (int32_t i = 0; i < N; ++i)
       r[i] = st->flags[i] != ORC_FLAG_EVICTABLE ? std::numeric_limits<float>::infinity()

@@ -32,7 +32,7 @@ extern "C" {
 #endif
 
 enum { ORC_FLAG_EVICTABLE = 0, ORC_FLAG_INIT = 1, ORC_FLAG_HIST = 2 };
-enum { ORC_SCORE_HYBRID = 0, ORC_SCORE_RESIDUAL_STORED = 1 };
+enum { ORC_SCORE_HYBRID = 0, ORC_SCORE_RESIDUAL_STORED = 1, ORC_SCORE_RANDOM = 2 };
 
 typedef struct {
   int32_t n_heads, head_dim;             /* C = n_heads * head_dim */
@@ -45,6 +45,7 @@ typedef struct {
   int32_t score_mode;                    /* ORC_SCORE_* */
   int32_t diversity_per_head;            /* 0: cosine on the whole C-vector; 1: mean over heads of per-head cosine */
   int32_t camera_cache;                  /* 1: the camera head's cache (Supp. C): one token per frame, grid 0 x 0 */
+  uint64_t random_seed;                  /* ORC_SCORE_RANDOM: seed of the per-step uniform priorities */
 } orc_config;
 
 typedef struct orc_state orc_state;
@@ -68,6 +69,16 @@ void orc_diversity(const float* K, int32_t n, int32_t C, int32_t n_heads, int32_
  * (flags != 0) take no part and get +inf.  r is fp32 [n + M]. */
 void orc_hybrid(const double* d, const double* s, const uint8_t* flags, int32_t n, int32_t M,
                 double beta, float* r);
+
+/* The random-eviction baseline of the paper's full-cache comparison (Supp. A): under the same budget, the rows that
+ * leave are drawn uniformly at random.  Here: every evictable row gets a fresh uniform priority in [0, 1) per step
+ * and Eq. 8 keeps the largest, which is a uniformly random subset.  The priority of token `token_id` in the step
+ * of frame `frame_id` is a counter-based value, so that both sides of a parity test can compute it:
+ *   u = top 24 bits of SplitMix64(SplitMix64(seed ^ frame_id) + token_id), scaled by 2^-24,
+ * SplitMix64(x) being one output step of that generator from state x (Steele, Lea, Flood 2014):
+ *   z = x + 0x9E3779B97F4A7C15; z = (z ^ z >> 30) * 0xBF58476D1CE4E5B9; z = (z ^ z >> 27) * 0x94D049BB133111EB; z ^ z >> 31. */
+uint64_t orc_splitmix64(uint64_t x);
+float orc_random_priority(uint64_t seed, int64_t frame_id, int64_t token_id);
 
 /* Eq. 8: keep every protected row and the (B - |P|) evictable rows of largest r;
  * ties go to the lower position, NaN ranks with -inf.  Returns the survivor

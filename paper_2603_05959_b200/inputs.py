@@ -26,6 +26,7 @@ DTYPE_BF16 = 1
 
 SCORE_HYBRID = 0
 SCORE_RESIDUAL_STORED = 1
+SCORE_RANDOM = 2
 
 
 @dataclasses.dataclass(frozen=True)

@@ -428,6 +428,63 @@ def test_stored_scores_travel_with_their_rows_through_every_compaction():
     assert len({int(i) // M for i in layer.export(with_kv=False)["ids"]}) >= 3
 
 
+# ------------------------------------------------------------------ Supp. A: the random-eviction baseline
+
+def test_splitmix64_reference_outputs_and_priority_range():
+    """The generator behind the random-eviction baseline against the published reference outputs of SplitMix64
+    (state 0: the first three outputs), and the priority against the formula written out with Python integers."""
+    golden = 0x9E3779B97F4A7C15
+    assert orc.splitmix64(0) == 0xE220A8397B1DCDAF
+    assert orc.splitmix64(golden) == 0x6E789E6AA1B965F4
+    assert orc.splitmix64(2 * golden) == 0x06C45D188009454F
+
+    def mix(x):
+        m = 2 ** 64 - 1
+        z = (x + golden) & m
+        z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & m
+        z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & m
+        return z ^ (z >> 31)
+
+    us = []
+    for seed, t, tok in [(0, 0, 0), (20260305, 7, 483), (2 ** 63 + 5, 9999, 13_739_999), (1, 2, 3)]:
+        want = (mix((mix(seed ^ t) + tok) & (2 ** 64 - 1)) >> 40) / 2.0 ** 24
+        got = orc.random_priority(seed, t, tok)
+        assert got == want and 0.0 <= got < 1.0
+        us.append(got)
+    assert len(set(us)) == 4
+    u = np.array([orc.random_priority(5, 3, i) for i in range(20000)])
+    assert abs(u.mean() - 0.5) < 0.01 and abs(np.mean(u < 0.1) - 0.1) < 0.01      # uniform, roughly
+
+
+def test_random_eviction_mode_keeps_a_uniform_subset_and_every_protected_row():
+    cfg = gen.config_tiny().replace(score_mode=gen.SCORE_RANDOM, budget=150, anchor_tokens=4, min_anchor_interval=3,
+                                    tau=0.9, n_frames=40)
+    layer = orc.OracleLayer.from_stream(cfg)
+    M = cfg.tokens_per_frame
+    evicted_pos = []
+    for t in range(cfg.n_frames):
+        fi = gen.frame_inputs(cfg, t)
+        layer.attend(t, fi.q, fi.k, fi.v, compute=False)
+        pre = layer.export(with_kv=False)
+        out = layer.compress(fi.resid, fi.conf, fi.rho)
+        fin = np.isfinite(out["r"])
+        want = np.array([orc.random_priority(cfg.seed, t, int(i)) for i in pre["ids"]], dtype=np.float32)
+        np.testing.assert_array_equal(out["r"][fin], want[fin])
+        # Eq. 8 on those priorities, by brute force
+        N = len(pre["ids"])
+        if N > cfg.budget:
+            prot = np.flatnonzero(~fin)
+            order = sorted(np.flatnonzero(fin), key=lambda i: (-out["r"][i], i))[: cfg.budget - len(prot)]
+            np.testing.assert_array_equal(out["survivors"], np.sort(np.concatenate([prot, order])))
+            gone = np.setdiff1d(np.arange(N), out["survivors"])
+            evicted_pos += (gone / N).tolist()
+        ex = layer.export(with_kv=False)
+        assert np.array_equal(ex["ids"][:M], np.arange(M))                       # the first frame stays
+    # evictions fall all over the buffer, old rows and new rows alike (a score-based rule would not do that)
+    hist = np.histogram(evicted_pos, bins=4, range=(0, 1))[0] / len(evicted_pos)
+    assert len(evicted_pos) > 1500 and hist[1:].min() > 0.15
+
+
 # ------------------------------------------------------------------ Supp. C: the camera head's cache
 
 def _camera_token(cfg, t, tag):
