@@ -58,7 +58,13 @@ enum {
 };
 
 enum { OVGGT_DTYPE_F32 = 0, OVGGT_DTYPE_BF16 = 1 };
-enum { OVGGT_SCORE_HYBRID = 0, OVGGT_SCORE_RESIDUAL_STORED = 1 };
+/* How evictable rows are ranked.  HYBRID is the paper's method (Eq. 7).  RESIDUAL_STORED ranks every row by the
+ * smoothed residual norm it had when new.  RANDOM is the random-eviction baseline of the paper's full-cache comparison
+ * (Supp. A): the rows that leave are drawn uniformly at random under the same budget - every evictable row gets a
+ * fresh uniform priority per step, the top 24 bits of SplitMix64(SplitMix64(random_seed ^ frame_id) + token_id)
+ * scaled by 2^-24 (SplitMix64(x): z = x + 0x9E3779B97F4A7C15; z = (z ^ z >> 30) * 0xBF58476D1CE4E5B9;
+ * z = (z ^ z >> 27) * 0x94D049BB133111EB; z ^ z >> 31), so that a run is reproducible from its seed. */
+enum { OVGGT_SCORE_HYBRID = 0, OVGGT_SCORE_RESIDUAL_STORED = 1, OVGGT_SCORE_RANDOM = 2 };
 enum { OVGGT_FLAG_EVICTABLE = 0, OVGGT_FLAG_INIT = 1, OVGGT_FLAG_HIST = 2 };
 /* Where surviving K/V rows live after Eq. 8 (the paper fixes the survivor set, not a layout):
  *  FILL_HOLES     one K/V buffer per layer; the rows admitted from the new frame are copied into the slots the
@@ -80,9 +86,10 @@ typedef struct {
   int32_t min_anchor_interval;           /* frames between anchor registrations (paper: 100) */
   float tau, alpha, beta;                /* coverage threshold, smoothing strength (Eq. 6), hybrid balance (Eq. 7) */
   int32_t protect_first_frame;           /* 1: Global Initial Anchor (all M first-frame tokens kept for good) */
-  int32_t score_mode;                    /* OVGGT_SCORE_HYBRID (Eq. 7) or OVGGT_SCORE_RESIDUAL_STORED */
+  int32_t score_mode;                    /* OVGGT_SCORE_* */
   int32_t dtype;                         /* OVGGT_DTYPE_* of q, k, v, resid, out and of the cache */
   int32_t compaction;                    /* OVGGT_COMPACT_* */
+  uint64_t random_seed;                  /* OVGGT_SCORE_RANDOM only */
   int32_t camera_head;                   /* 1: the camera head's cache (Supp. C): n_special = 1, grid 0 x 0,
                                             anchor_tokens = 0; see ovggt_camera_compress.  0: an aggregator cache */
   void* workspace;                       /* device, >= ovggt_workspace_bytes(cfg), 1024-byte aligned; need not be zeroed */
@@ -142,6 +149,16 @@ int ovggt_layer_attend(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* 
  * score_override. */
 int ovggt_layer_compress(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
 
+/* ovggt_layer_compress for every layer of the handle in one call (Sec. 3.2: each layer l has its own budget B^(l),
+ * given at create): ios [n_ios], n_ios = n_layers, ios[l] describing layer l's pending frame (all with the same
+ * frame_id; conf and rho are taken from ios[0]).  This is the call for a model whose anchor inputs exist only after
+ * its heads have run: attend layer by layer, then compress all layers together.  In the hole-filling layout the
+ * scores, the selection and the moves of up to 32 layers each go out as one launch (blockIdx.y = layer; one
+ * thread-block cluster per layer for the selection), so the small per-layer kernels fill the GPU together; in the
+ * stable-gather layout the layers are compressed one after the other.  All layers are checked before anything
+ * changes; results are those of n_layers single calls. */
+int ovggt_layers_compress(ovggt_cache* cache, const ovggt_frame_io* ios, int32_t n_ios, void* stream);
+
 /* Supp. C: the camera prediction head keeps one token per frame in a cache of its own, under the same scoring and
  * protection.  Create it as a second handle with camera_head = 1 (budget[l] >= 1 + K_max tokens), run
  * ovggt_layer_attend on it with the camera token's q, k, v ([1, C]), and compress it with this call instead of
@@ -167,6 +184,14 @@ int ovggt_layer_step(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io
 /* Turn the overlap of ovggt_layer_step off (0) or on (non-zero, the default): off, the two halves run one after the
  * other on `stream`, which is what per-kernel timing wants. */
 int ovggt_cache_set_overlap(ovggt_cache* cache, int32_t enable);
+
+/* The bf16 attention kernel may take a softmax reference that needs no tracking: per layer the library keeps a
+ * running upper bound of the per-head key norms (updated by every append, recomputed by an import, cleared by a
+ * reset; it never shrinks, so it stays a bound when keys are evicted), and |q| |k|_max / sqrt(64) bounds every logit
+ * of a query row.  A warp whose 32 rows all find that bound within 2^48 of the true maximum of their first 96 scores
+ * uses it for good and skips maximum tracking and rescaling; other warps track the maximum as before.  Results agree
+ * within the attention tolerance either way.  On by default; 0 turns it off for the handle. */
+int ovggt_cache_set_key_bound(ovggt_cache* cache, int32_t enable);
 
 /* The same step with HOST tensors: q, k, v, resid, conf, out are host pointers; score_override must be NULL.
  * The host inputs must hold their values when the call is made.  They are copied into one of two sets of staging
@@ -293,6 +318,14 @@ int ovggt_k_compact(const void* k_src, const void* v_src, const int32_t* survivo
 size_t ovggt_k_attention_scratch_bytes(int32_t M, int32_t N, int32_t n_heads);
 int ovggt_k_attention(const void* q, const void* k, const void* v, int32_t M, int32_t N, int32_t n_heads,
                       int32_t dtype, void* out, void* scratch, int32_t* device_status, void* stream);
+
+/* The bf16 attention with a fixed softmax reference where it is safe (see ovggt_cache_set_key_bound).
+ * ovggt_k_key_norm_bound: kmax2 [n_heads] (device) = max over the rows of K [rows, n_heads * 64] (bf16) of the squared
+ * norm of each head's 64 columns; n_heads <= 16.  ovggt_k_attention_bounded: as ovggt_k_attention for bf16, given such
+ * a bound for (at least) the N keys it attends over; a bound that is too small voids the result. */
+int ovggt_k_key_norm_bound(const void* K, int32_t rows, int32_t n_heads, float* kmax2, void* stream);
+int ovggt_k_attention_bounded(const void* q, const void* k, const void* v, int32_t M, int32_t N, int32_t n_heads,
+                              void* out, void* scratch, int32_t* device_status, const float* kmax2, void* stream);
 
 #ifdef __cplusplus
 }

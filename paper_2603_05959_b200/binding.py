@@ -17,20 +17,20 @@ LIB_PATH = os.path.join(_HERE, "libovggt.so")
 MAX_ANCHORS = 16
 
 DTYPE_F32, DTYPE_BF16 = 0, 1
-SCORE_HYBRID, SCORE_RESIDUAL_STORED = 0, 1
+SCORE_HYBRID, SCORE_RESIDUAL_STORED, SCORE_RANDOM = 0, 1, 2
 FLAG_EVICTABLE, FLAG_INIT, FLAG_HIST = 0, 1, 2
 COMPACT_FILL_HOLES, COMPACT_STABLE_GATHER = 0, 1
 PROF_CLASSES = ["append", "attention", "row_norms", "diversity", "select", "compact"]
 
 EXPORTED = [
     "ovggt_workspace_bytes", "ovggt_cache_create", "ovggt_cache_destroy", "ovggt_layer_attend",
-    "ovggt_layer_compress", "ovggt_layer_step", "ovggt_layer_step_host", "ovggt_cache_stats",
+    "ovggt_layer_compress", "ovggt_layers_compress", "ovggt_layer_step", "ovggt_layer_step_host", "ovggt_cache_stats",
     "ovggt_cache_export", "ovggt_cache_import", "ovggt_cache_reset", "ovggt_cache_anchor_decision",
     "ovggt_camera_compress", "ovggt_cache_selftest_bounded_wait", "ovggt_cache_clear_status", "ovggt_cache_last_selection", "ovggt_kernel_launches",
-    "ovggt_cache_profile_enable", "ovggt_cache_profile_read", "ovggt_cache_set_overlap",
+    "ovggt_cache_profile_enable", "ovggt_cache_profile_read", "ovggt_cache_set_overlap", "ovggt_cache_set_key_bound",
     "ovggt_strerror", "ovggt_last_cuda_error", "ovggt_k_row_norms", "ovggt_k_diversity_scratch_bytes",
     "ovggt_k_diversity", "ovggt_k_diversity_static", "ovggt_k_select", "ovggt_k_compact", "ovggt_k_attention_scratch_bytes",
-    "ovggt_k_attention",
+    "ovggt_k_attention", "ovggt_k_key_norm_bound", "ovggt_k_attention_bounded",
 ]
 
 
@@ -42,7 +42,7 @@ class OvggtConfig(C.Structure):
         ("anchor_tokens", C.c_int32), ("k_max", C.c_int32), ("min_anchor_interval", C.c_int32),
         ("tau", C.c_float), ("alpha", C.c_float), ("beta", C.c_float),
         ("protect_first_frame", C.c_int32), ("score_mode", C.c_int32), ("dtype", C.c_int32),
-        ("compaction", C.c_int32), ("camera_head", C.c_int32),
+        ("compaction", C.c_int32), ("random_seed", C.c_uint64), ("camera_head", C.c_int32),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
     ]
 
@@ -89,8 +89,9 @@ def lib():
         L.ovggt_workspace_bytes.argtypes = [C.POINTER(OvggtConfig)]
         L.ovggt_cache_create.argtypes = [C.POINTER(OvggtConfig), C.POINTER(vp)]
         L.ovggt_cache_destroy.argtypes = [vp]
-        for name in ("ovggt_layer_attend", "ovggt_layer_compress", "ovggt_layer_step", "ovggt_layer_step_host"):
+        for name in ("ovggt_layer_attend", "ovggt_layer_compress", "ovggt_layers_compress", "ovggt_layer_step", "ovggt_layer_step_host"):
             getattr(L, name).argtypes = [vp, i32, C.POINTER(OvggtFrameIO), vp]
+        L.ovggt_layers_compress.argtypes = [vp, C.POINTER(OvggtFrameIO), i32, vp]
         L.ovggt_cache_stats.argtypes = [vp, i32, C.POINTER(OvggtStats)]
         L.ovggt_cache_export.argtypes = [vp, i32, vp, vp, vp, vp, vp, C.POINTER(i32)]
         L.ovggt_cache_import.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32, i64, i64]
@@ -102,6 +103,7 @@ def lib():
         L.ovggt_cache_last_selection.argtypes = [vp, i32, vp, C.POINTER(i32), vp, C.POINTER(i32)]
         L.ovggt_cache_profile_enable.argtypes = [vp, i32]
         L.ovggt_cache_set_overlap.argtypes = [vp, i32]
+        L.ovggt_cache_set_key_bound.argtypes = [vp, i32]
         L.ovggt_cache_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_int64), i32]
         L.ovggt_kernel_launches.restype = C.c_uint64
         L.ovggt_strerror.restype = C.c_char_p
@@ -116,6 +118,8 @@ def lib():
         L.ovggt_k_attention_scratch_bytes.restype = C.c_size_t
         L.ovggt_k_attention_scratch_bytes.argtypes = [i32, i32, i32]
         L.ovggt_k_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
+        L.ovggt_k_key_norm_bound.argtypes = [vp, i32, i32, vp, vp]
+        L.ovggt_k_attention_bounded.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
         _LIB = L
     return _LIB
 
@@ -157,13 +161,14 @@ class OvggtCache:
     def __init__(self, *, n_layers=1, n_heads=16, head_dim=64, n_special=5, grid_h=37, grid_w=37,
                  budget=16384, anchor_tokens=64, k_max=3, min_anchor_interval=100, tau=0.2, alpha=0.5,
                  beta=0.5, protect_first_frame=1, score_mode=SCORE_HYBRID, dtype=DTYPE_BF16,
-                 compaction=COMPACT_FILL_HOLES, camera_head=0, device: Optional[torch.device] = None):
+                 compaction=COMPACT_FILL_HOLES, random_seed=0, camera_head=0,
+                 device: Optional[torch.device] = None):
         budgets = [budget] * n_layers if isinstance(budget, int) else list(budget)
         assert len(budgets) == n_layers
         self._budgets = (C.c_int32 * n_layers)(*budgets)
         self.cfg = OvggtConfig(n_layers, n_heads, head_dim, n_special, grid_h, grid_w, self._budgets,
                                anchor_tokens, k_max, min_anchor_interval, tau, alpha, beta,
-                               protect_first_frame, score_mode, dtype, compaction, camera_head, None, 0)
+                               protect_first_frame, score_mode, dtype, compaction, random_seed, camera_head, None, 0)
         self.compaction = compaction
         self.M = n_special + grid_h * grid_w
         self.C = n_heads * head_dim
@@ -194,7 +199,7 @@ class OvggtCache:
                   anchor_tokens=cfg.anchor_tokens, k_max=cfg.k_max,
                   min_anchor_interval=cfg.min_anchor_interval, tau=cfg.tau, alpha=cfg.alpha,
                   beta=cfg.beta, protect_first_frame=cfg.protect_first_frame,
-                  score_mode=cfg.score_mode, dtype=cfg.dtype)
+                  score_mode=cfg.score_mode, dtype=cfg.dtype, random_seed=cfg.seed)
         kw.update(over)
         return cls(**kw)
 
@@ -228,6 +233,15 @@ class OvggtCache:
                        stream=None) -> None:
         io = self._io(frame_id, resid=resid, conf=conf, rho=rho, score_override=score_override)
         _check(lib().ovggt_layer_compress(self._h, layer, C.byref(io), _stream_ptr(stream)), "ovggt_layer_compress")
+
+    def layers_compress(self, frame_id, resids, conf=None, rho=float("nan"), score_overrides=None, stream=None) -> None:
+        """ovggt_layers_compress: resids[l] (and optionally score_overrides[l]) per layer, one call for all layers."""
+        n = len(resids)
+        ios = (OvggtFrameIO * n)()
+        for l in range(n):
+            ov = None if score_overrides is None else score_overrides[l]
+            ios[l] = self._io(frame_id, resid=resids[l], conf=conf, rho=rho, score_override=ov)
+        _check(lib().ovggt_layers_compress(self._h, ios, n, _stream_ptr(stream)), "ovggt_layers_compress")
 
     def anchor_decision(self, frame_id):
         """(registered, demoted_frame) of frame_id as this (aggregator) handle decided it."""
@@ -303,6 +317,9 @@ class OvggtCache:
     def reset(self) -> None:
         _check(lib().ovggt_cache_reset(self._h), "ovggt_cache_reset")
 
+    def set_key_bound(self, on: bool) -> None:
+        _check(lib().ovggt_cache_set_key_bound(self._h, int(on)), "ovggt_cache_set_key_bound")
+
     def set_overlap(self, on: bool) -> None:
         _check(lib().ovggt_cache_set_overlap(self._h, int(on)), "ovggt_cache_set_overlap")
 
@@ -376,10 +393,28 @@ def k_compact(k_src, v_src, survivors, k_dst=None, v_dst=None, stream=None):
     return k_dst, v_dst
 
 
-def k_attention(q, k, v, n_heads: int, out=None, scratch=None, status=None, stream=None) -> torch.Tensor:
+def k_key_norm_bound(k: torch.Tensor, n_heads: int, stream=None) -> torch.Tensor:
+    """[n_heads] fp32: the largest squared norm of any key's 64 columns of each head (bf16 keys)."""
+    out = torch.empty(n_heads, dtype=torch.float32, device=k.device)
+    _check(lib().ovggt_k_key_norm_bound(_dptr(k), k.shape[0], n_heads, _dptr(out), _stream_ptr(stream)),
+           "ovggt_k_key_norm_bound")
+    return out
+
+
+def k_attention(q, k, v, n_heads: int, out=None, scratch=None, status=None, stream=None, bounded=False) -> torch.Tensor:
+    """bounded: bf16 only - first compute the key-norm bound, then attend with the fixed softmax reference."""
     dtype = DTYPE_F32 if q.dtype == torch.float32 else DTYPE_BF16
     M, N = q.shape[0], k.shape[0]
     out = torch.empty_like(q) if out is None else out
+    if bounded:
+        assert dtype == DTYPE_BF16
+        kmax2 = k_key_norm_bound(k, n_heads, stream)
+        scratch = torch.empty(lib().ovggt_k_attention_scratch_bytes(M, N, n_heads), dtype=torch.uint8, device=q.device)
+        st = torch.zeros(16, dtype=torch.int32, device=q.device)
+        _check(lib().ovggt_k_attention_bounded(_dptr(q), _dptr(k), _dptr(v), M, N, n_heads, _dptr(out), _dptr(scratch),
+                                               _dptr(st), _dptr(kmax2), _stream_ptr(stream)), "ovggt_k_attention_bounded")
+        _check(int(st[0].item()), "ovggt_k_attention_bounded (device status)")
+        return out
     if scratch is None:
         scratch = torch.empty(lib().ovggt_k_attention_scratch_bytes(M, N, n_heads), dtype=torch.uint8, device=q.device)
     own_status = status is None

@@ -46,7 +46,15 @@ constexpr int kHalf = kBN / 2;      // KV rows per S buffer
 constexpr int kTmemCols = 256;
 constexpr int kColS = 0, kColO = 2 * kHalf;   // S_0 at columns [0, 96), S_1 at [96, 192), O at [192, 256): all 256 columns
 constexpr float kRescaleThreshold = 8.0f;          // log2 units
-constexpr int kPolyEvery = 4;                      // one pair of exponentials in kPolyEvery goes to the FMA pipes
+// A row whose logits have a known upper bound (|q| x the largest |k| of the cache, Cauchy-Schwarz) may take that bound
+// as its softmax reference for good: nothing can outgrow it, so the maximum need not be tracked and O never rescaled.
+// The price is that every exponential comes out 2^-(bound - true maximum) smaller than it could; fp32 sums and bf16
+// probabilities keep their relative precision as long as that stays far from the underflow threshold (2^-126).
+constexpr float kFixedRefMaxGap = 48.0f;           // log2 units between the bound and the first half's true maximum
+#ifndef OVGGT_ATTN_POLY_EVERY
+#define OVGGT_ATTN_POLY_EVERY 4
+#endif
+constexpr int kPolyEvery = OVGGT_ATTN_POLY_EVERY;  // one pair of exponentials in kPolyEvery goes to the FMA pipes
 constexpr int kMaxSplits = 16;
 
 struct AttnBarriers {
@@ -262,6 +270,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 struct AttnParams {
   int M, N, H;
   int splits, tiles_per_split, tiles_total;
+  const float* kmax2;     // [H] upper bound of |k_j,h|^2 over all N keys, or nullptr (the maximum is tracked)
   __nv_bfloat16* out;     // [M, C]            (splits == 1)
   float* o_part;          // [splits, M, C]    un-normalised partial outputs
   float2* ml_part;        // [splits, M, H]    (reference maximum in log2 units, row sum)
@@ -450,7 +459,29 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const float c = 1.4426950408889634f * 0.125f;     // log2(e) / sqrt(64)
     float mref = 0.0f, l = 0.0f;
     bool ok = true;
-    for (int idx = 0; idx < 2 * n_tiles; ++idx) {       // idx = 2 * tile + half
+    // Upper bound of this row's logits in log2 units: |q_row,h| |k|_max log2(e) / 8.  The row's 64 query values are
+    // the eight 16-byte chunks of its 128-byte line in the (swizzled) Q tile, in whatever order.
+    float bound = 0.0f;
+    bool fixed_ref = false;
+    if (P.kmax2 != nullptr) {
+      ok = __all_sync(0xFFFFFFFFu, mbar_wait(&B->q_full, 0, B, P.status)) != 0;
+      if (ok) {
+        float qn2 = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint4 u = *reinterpret_cast<const uint4*>(sQ + row * 128 + ((j ^ (row & 7)) << 4));
+          const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xFFFF0000u);
+            qn2 = fmaf(lo, lo, qn2);
+            qn2 = fmaf(hi, hi, qn2);
+          }
+        }
+        bound = sqrtf(qn2 * __ldg(P.kmax2 + h)) * c;
+      }
+    }
+    for (int idx = 0; idx < 2 * n_tiles && ok; ++idx) {       // idx = 2 * tile + half
       const int it = idx >> 1, hf = idx & 1;
       // (every wait result is made warp-uniform before the warp meets an .aligned tensor-memory instruction)
       ok = __all_sync(0xFFFFFFFFu, mbar_wait(&B->s_full[hf], (uint32_t)it & 1u, B, P.status)) != 0;
@@ -507,7 +538,19 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             m4[q] = max3(m4[q], __uint_as_float(s[kChain * q + j]), __uint_as_float(s[kChain * q + j + 1]));
         }
         mref = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * c;
+        if (P.kmax2 != nullptr) {
+          // take the bound as the reference if it is a bound for what was seen and not absurdly far above it; the
+          // decision is per warp, so that the warp stays in step
+          const bool safe = bound >= mref && bound - mref <= kFixedRefMaxGap;
+          fixed_ref = __all_sync(0xFFFFFFFFu, safe) != 0;
+          // a whole number of powers of two above the true maximum of this half: its largest probability is then an
+          // exact power of two, as it is (2^0) when the maximum itself is the reference, so a row that one early key
+          // dominates loses nothing to the bf16 rounding of P
+          if (fixed_ref) mref += ceilf(bound - mref);
+        }
         add = exp_pass(std::false_type{}, raw);
+      } else if (fixed_ref) {
+        add = exp_pass(std::false_type{}, raw);          // no score can exceed the reference: nothing to track
       } else {
         // Later halves compute p under the reference they inherit while the maximum is gathered, and keep the
         // result unless the maximum outgrew the reference by more than the threshold (rare); then O is rescaled,
@@ -742,7 +785,7 @@ inline int attn_kv_maps(AttnKvMaps* m, const void* k, const void* v, int N, int 
 
 inline int attn_tcgen05_launch(const void* q, const void* k, const void* v, int M, int N, int H, void* out,
                                void* scratch, int* status, cudaStream_t st, AttnKvMaps* kv_maps = nullptr,
-                               int force_splits = 0) {
+                               int force_splits = 0, const float* kmax2 = nullptr) {
   const int C = H * kHD;
   CUtensorMap tq;
   AttnKvMaps local;
@@ -763,6 +806,7 @@ inline int attn_tcgen05_launch(const void* q, const void* k, const void* v, int 
   P.o_part = static_cast<float*>(scratch);
   P.ml_part = reinterpret_cast<float2*>(static_cast<char*>(scratch) + (size_t)kMaxSplits * M * C * 4);
   P.status = status;
+  P.kmax2 = kmax2;
   cudaError_t e = cudaFuncSetAttribute(k_attn_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
   if (e != cudaSuccess) { g_attn_last_error = (int)e; return OVGGT_ERR_CUDA; }
   dim3 grid((M + kBM - 1) / kBM, H, P.splits);

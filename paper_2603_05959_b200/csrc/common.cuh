@@ -59,6 +59,19 @@ __device__ __forceinline__ uint32_t rank_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// One output step of the SplitMix64 generator from state x (Steele, Lea, Flood 2014), and the uniform priority in
+// [0, 1) that the random-eviction mode gives token `token_id` in the step of frame `frame_id`: the top 24 bits of
+// SplitMix64(SplitMix64(seed ^ frame_id) + token_id), exact in fp32.
+__host__ __device__ __forceinline__ unsigned long long splitmix64(unsigned long long x) {
+  unsigned long long z = x + 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+__host__ __device__ __forceinline__ float random_priority(unsigned long long step_key, long long token_id) {
+  return (float)(splitmix64(step_key + (unsigned long long)token_id) >> 40) * (1.0f / 16777216.0f);
+}
+
 // ---- block-wide primitives for a block of up to 1024 threads; `sh` holds >= 33 words.
 
 __device__ inline int block_sum_int(int x, int* sh) {

@@ -116,20 +116,75 @@ __global__ void __launch_bounds__(256) k_compact_colsum(const uint4* __restrict_
     part[(size_t)blockIdx.x * C + c] = ((red[0][c] + red[1][c]) + red[2][c]) + red[3][c];
 }
 
+// Running upper bound of the squared per-head key norms of a bf16 cache, head_dim 64: kmax2[h] = max(kmax2[h],
+// |K[row, 64h .. 64h+63]|^2).  A warp holds the row as 16-byte vectors (lane + 32 i); a head is eight consecutive
+// vectors, i.e. eight neighbouring lanes of one i.  Non-negative floats order like their bit patterns, so the maximum
+// is an integer atomicMax, which does not depend on the order of arrival.
+__device__ __forceinline__ void warp_key_norm_max(const uint4* u, int nvec, int lane, float* kmax2) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float ss = 0.0f;
+    if (lane + 32 * i < nvec) {
+      const uint32_t w[4] = {u[i].x, u[i].y, u[i].z, u[i].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float lo = __uint_as_float(w[e] << 16), hi = __uint_as_float(w[e] & 0xFFFF0000u);
+        ss = fmaf(lo, lo, ss);
+        ss = fmaf(hi, hi, ss);
+      }
+    }
+    ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
+    ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
+    ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 4);
+    if ((lane & 7) == 0 && lane + 32 * i < nvec) {
+      const int head = (lane + 32 * i) >> 3;
+      if (ss > kmax2[head]) atomicMax(reinterpret_cast<int*>(kmax2) + head, __float_as_int(ss));
+    }
+  }
+}
+
+// kmax2 over rows [0, rows) of K (after an import).  bf16, nvec <= 128.
+__global__ void __launch_bounds__(256) k_key_norm_max(const uint4* __restrict__ K, int rows, int nvec,
+                                                      float* __restrict__ kmax2) {
+  const int lane = threadIdx.x & 31;
+  const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
+  for (int r = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5); r < rows; r += warps_total) {
+    uint4 u[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (lane + 32 * i < nvec) u[i] = ld_nc(K + (size_t)r * nvec + lane + 32 * i);
+    warp_key_norm_max(u, nvec, lane, kmax2);
+  }
+}
+
 // Rows [n, n+M) of the cache := the frame's K and V; their meta: ids frame*M + j, evictable, score 0 and, in the
-// hole-filling layout (slot != nullptr), the physical slot n + j.
+// hole-filling layout (slot != nullptr), the physical slot n + j.  With kmax2 (bf16 rows of up to 128 vectors) the
+// running bound of the key norms takes the new keys in.
 __global__ void __launch_bounds__(256) k_append(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new,
                                                 int M, int nvec, int n, long long frame_id,
                                                 uint4* __restrict__ k_cache, uint4* __restrict__ v_cache,
                                                 long long* __restrict__ ids, uint8_t* __restrict__ flags,
-                                                float* __restrict__ stored, int* __restrict__ slot) {
+                                                float* __restrict__ stored, int* __restrict__ slot,
+                                                float* __restrict__ kmax2) {
   const int lane = threadIdx.x & 31;
   const int gtid = blockIdx.x * blockDim.x + threadIdx.x;
   const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
   for (int item = gtid >> 5; item < 2 * M; item += warps_total) {
     const int j = item >> 1;
-    if (item & 1) warp_copy_row(v_new + (size_t)j * nvec, v_cache + (size_t)(n + j) * nvec, nvec, lane);
-    else          warp_copy_row(k_new + (size_t)j * nvec, k_cache + (size_t)(n + j) * nvec, nvec, lane);
+    if (item & 1) {
+      warp_copy_row(v_new + (size_t)j * nvec, v_cache + (size_t)(n + j) * nvec, nvec, lane);
+    } else if (kmax2 == nullptr) {
+      warp_copy_row(k_new + (size_t)j * nvec, k_cache + (size_t)(n + j) * nvec, nvec, lane);
+    } else {
+      uint4 u[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (lane + 32 * i < nvec) u[i] = ld_nc(k_new + (size_t)j * nvec + lane + 32 * i);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (lane + 32 * i < nvec) k_cache[(size_t)(n + j) * nvec + lane + 32 * i] = u[i];
+      warp_key_norm_max(u, nvec, lane, kmax2);
+    }
   }
   for (int j = gtid; j < M; j += gridDim.x * blockDim.x) {
     ids[n + j] = frame_id * (long long)M + j;

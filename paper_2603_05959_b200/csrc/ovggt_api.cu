@@ -226,9 +226,10 @@ int launch_fill_holes(void* kc, void* vc, const int* msrc, const int* mdst, cons
 }
 
 int launch_attention(const void* q, const void* k, const void* v, int M, int N, int H, int dtype, void* out,
-                     void* scratch, int* status, cudaStream_t st, AttnKvMaps* maps = nullptr) {
+                     void* scratch, int* status, cudaStream_t st, AttnKvMaps* maps = nullptr,
+                     const float* kmax2 = nullptr) {
   if (dtype == kBF16) {
-    int rc = attn_tcgen05_launch(q, k, v, M, N, H, out, scratch, status, st, maps);
+    int rc = attn_tcgen05_launch(q, k, v, M, N, H, out, scratch, status, st, maps, 0, kmax2);
     if (rc == OVGGT_OK) g_launches.fetch_add(attn_tcgen05_num_launches(M, N, H));
     if (rc == OVGGT_ERR_CUDA) g_last_cuda_error.store(attn_tcgen05_last_error());
     return rc;
@@ -274,6 +275,7 @@ struct LayerState {
   int kcur = 0;                   // which of the two the next diversity launch reads
   bool ksum_valid = false;        // ksum[kcur] describes the cached keys (else: recompute)
   int since_refresh = 0;
+  float* kmax2 = nullptr;         // [n_heads] running upper bound of the squared per-head key norms (bf16 caches)
   AttnKvMaps maps[2];             // tensor maps of the K/V buffers, re-encoded only when the row count changes
   int64_t scores_frame = -1;      // frame whose s_raw and d were already enqueued on the side stream
   size_t kv_bytes = 0;
@@ -309,6 +311,7 @@ struct ovggt_cache {
   cudaStream_t side = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_app = nullptr;
   bool overlap = true;            // ovggt_cache_set_overlap
+  bool use_key_bound = true;      // ovggt_cache_set_key_bound
   // optional per-kernel-class timing (host-side CUDA events; no device memory)
   bool prof = false;
   struct ProfRec { int cls; cudaEvent_t a, b; };
@@ -363,7 +366,9 @@ bool config_ok(const ovggt_config* c, int* err) {
   if (c->anchor_tokens < 0 || c->anchor_tokens > c->grid_h * c->grid_w) return false;
   if (c->k_max < 0 || c->k_max > OVGGT_MAX_ANCHORS || c->min_anchor_interval < 0) return false;
   if (c->dtype != kF32 && c->dtype != kBF16) return false;
-  if (c->score_mode != OVGGT_SCORE_HYBRID && c->score_mode != OVGGT_SCORE_RESIDUAL_STORED) return false;
+  if (c->score_mode != OVGGT_SCORE_HYBRID && c->score_mode != OVGGT_SCORE_RESIDUAL_STORED &&
+      c->score_mode != OVGGT_SCORE_RANDOM)
+    return false;
   if (c->compaction != OVGGT_COMPACT_FILL_HOLES && c->compaction != OVGGT_COMPACT_STABLE_GATHER) return false;
   if (!(c->alpha >= 0.0f && c->alpha <= 1.0f) || !(c->beta >= 0.0f && c->beta <= 1.0f)) return false;
   const int64_t M = c->n_special + (int64_t)c->grid_h * c->grid_w;
@@ -411,6 +416,7 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
     off[i++] = L.take(R * 4);           // r
     off[i++] = L.take(R * 4);           // survivors
     off[i++] = L.take(64);              // n_keep, n_moves
+    off[i++] = L.take((size_t)c->n_heads * 4);   // bound of the key norms
     if (fill) {
       for (int b = 0; b < 2; ++b) off[i++] = L.take(R * 4);                                  // slots
       for (int b = 0; b < 3; ++b) off[i++] = L.take((size_t)M * 4);                          // move lists
@@ -433,6 +439,7 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
       S.surv = reinterpret_cast<int*>(base + off[i++]);
       S.n_keep_dev = reinterpret_cast<int*>(base + off[i++]);
       S.n_moves_dev = S.n_keep_dev + 4;
+      S.kmax2 = reinterpret_cast<float*>(base + off[i++]);
       if (fill) {
         for (int b = 0; b < 2; ++b) S.slot[b] = reinterpret_cast<int*>(base + off[i++]);
         S.move_src = reinterpret_cast<int*>(base + off[i++]);
@@ -546,6 +553,8 @@ extern "C" int ovggt_cache_create(const ovggt_config* cfg, ovggt_cache** out) {
   }
   cudaError_t e = cudaMemset(h->status, 0, 64);
   if (e == cudaSuccess) e = cudaMemset(h->ksum, 0, colsum_scratch_bytes(h->C));   // (its arrival counters)
+  for (LayerState& S : h->layers)
+    if (e == cudaSuccess) e = cudaMemset(S.kmax2, 0, (size_t)cfg->n_heads * 4);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     delete h;
@@ -596,6 +605,13 @@ int validate_attend(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io) {
   return OVGGT_OK;
 }
 
+// The bound of the key norms is kept for bf16 caches whose rows the append kernel holds in one round of loads; the
+// attention kernel then takes |q| |k|_max as a fixed softmax reference.  It only grows (evictions do not lower it),
+// which keeps it a bound; ovggt_cache_reset clears it, an import recomputes it.
+float* key_norm_bound(const ovggt_cache* h, const LayerState& S) {
+  return (h->cfg.dtype == kBF16 && h->C * h->elem / 16 <= 128 && h->use_key_bound) ? S.kmax2 : nullptr;
+}
+
 // Eq. 2: the append itself.
 int enqueue_append(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st) {
   int rc = validate_attend(h, layer, io);
@@ -606,7 +622,8 @@ int enqueue_append(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cuda
   const int grid = std::min((2 * M + 7) / 8, 148 * 8);
   ProfScope ps(h, OVGGT_PROF_APPEND, st);
   k_append<<<grid, 256, 0, st>>>((const uint4*)io->k, (const uint4*)io->v, M, nvec, S.n, (long long)io->frame_id,
-                                 (uint4*)S.kbuf[kb], (uint4*)S.vbuf[kb], S.ids[b], S.flags[b], S.stored[b], S.slot[b]);
+                                 (uint4*)S.kbuf[kb], (uint4*)S.vbuf[kb], S.ids[b], S.flags[b], S.stored[b], S.slot[b],
+                                 key_norm_bound(h, S));
   LAUNCHED();
   return OVGGT_OK;
 }
@@ -620,7 +637,7 @@ int enqueue_attention(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, c
   {
     ProfScope ps(h, OVGGT_PROF_ATTENTION, st);
     rc = launch_attention(io->q, S.kbuf[kb], S.vbuf[kb], h->M, S.n + h->M, h->cfg.n_heads, h->cfg.dtype, io->out,
-                          h->attn_scratch, h->status, st, &S.maps[kb]);
+                          h->attn_scratch, h->status, st, &S.maps[kb], key_norm_bound(h, S));
   }
   if (rc) return rc;
   if (h->first_frame < 0) {
@@ -674,77 +691,69 @@ int enqueue_scores(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io, cuda
   return launch_diversity(S.kbuf[kb], n, C, c.dtype, h->colsum_part, h->ksum, S.d, st);
 }
 
-// The compress half.  Scores and selection go to st_sel.  What moves K/V rows goes to st_move: the stable gather
-// writes another buffer and may run beside an attention that still reads this one (st_move = st_sel); the
-// hole-filling move writes the buffer the attention reads, so it follows both (st_move = the attention's stream,
-// which first waits for st_sel).
 // `mirrored`: the anchor decision of the frame as another handle took it (camera head, Supp. C) instead of the rule
 // of Sec. 3.3 applied to rho.
 struct MirroredDecision { bool registered; int64_t demoted_frame; };
 
-int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st_sel, cudaStream_t st_move,
-                  const MirroredDecision* mirrored = nullptr) {
+// Argument and order checks of the compress half; nothing is changed.
+int validate_compress(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, const MirroredDecision* mirrored) {
   int rc = check_layer(h, layer);
   if (rc) return rc;
   if (!io || !io->resid) return OVGGT_ERR_INVALID_ARG;
   if ((h->cfg.camera_head != 0) != (mirrored != nullptr)) return OVGGT_ERR_INVALID_ARG;
   if (!aligned16(io->resid)) return OVGGT_ERR_MISALIGNED;
-  LayerState& S = h->layers[layer];
+  const LayerState& S = h->layers[layer];
   if (!S.pending || io->frame_id != S.pending_frame) return OVGGT_ERR_FRAME_ORDER;
-  const ovggt_config& c = h->cfg;
-  const int M = h->M, C = h->C, n = S.n, N = n + M, B = S.budget, b = S.cur, kb = S.kv;
-  const int64_t t = io->frame_id;
-  const bool fill = fill_layout(h);
-  const int ncta = select_cluster_ctas(N);
-  const size_t smem = compress_smem_bytes((N + ncta - 1) / ncta, h->Np, M);
-  if (smem > kSmemLimit) return OVGGT_ERR_UNSUPPORTED;   // (create already refuses such budgets)
+  const int N = S.n + h->M, ncta = select_cluster_ctas(N);
+  if (compress_smem_bytes((N + ncta - 1) / ncta, h->Np, h->M) > kSmemLimit)
+    return OVGGT_ERR_UNSUPPORTED;   // (create already refuses such budgets)
   // The anchor state belongs to the whole handle and moves forward only: a layer that comes with a frame older
   // than the last decision would take that frame's decision a second time.
-  if (t < h->decided_frame) return OVGGT_ERR_FRAME_ORDER;
+  if (io->frame_id < h->decided_frame) return OVGGT_ERR_FRAME_ORDER;
+  return OVGGT_OK;
+}
 
-  // Anchor decision of this frame (Sec. 3.3), taken once and shared by all layers; nothing below can fail on
-  // an argument any more.
-  if (h->decided_frame != t) {
-    h->decided_frame = t;
-    h->decided_register = false;
-    h->decided_demote = -1;
-    if (mirrored) {
-      // the frame's token is protected / the demoted frame's token released exactly when the aggregator did so
-      if (t != h->first_frame && mirrored->registered && (int)h->anchors.size() < OVGGT_MAX_ANCHORS) {
-        h->decided_register = true;
-        h->anchors.push_back(t);
-        h->last_registration = t;
-      }
-      if (mirrored->demoted_frame >= 0) {
-        auto it = std::find(h->anchors.begin(), h->anchors.end(), mirrored->demoted_frame);
-        if (it != h->anchors.end()) {
-          h->decided_demote = mirrored->demoted_frame;
-          h->anchors.erase(it);
-        }
-      }
-    } else if (t != h->first_frame && c.anchor_tokens > 0 && c.k_max > 0 && io->conf != nullptr && io->rho < c.tau &&
-               t - h->last_registration >= c.min_anchor_interval) {
+// Anchor decision of frame t (Sec. 3.3), taken once and shared by all layers.
+void take_decision(ovggt_cache* h, const ovggt_frame_io* io, const MirroredDecision* mirrored) {
+  const ovggt_config& c = h->cfg;
+  const int64_t t = io->frame_id;
+  if (h->decided_frame == t) return;
+  h->decided_frame = t;
+  h->decided_register = false;
+  h->decided_demote = -1;
+  if (mirrored) {
+    // the frame's token is protected / the demoted frame's token released exactly when the aggregator did so
+    if (t != h->first_frame && mirrored->registered && (int)h->anchors.size() < OVGGT_MAX_ANCHORS) {
       h->decided_register = true;
       h->anchors.push_back(t);
       h->last_registration = t;
-      if ((int)h->anchors.size() > c.k_max) {
-        h->decided_demote = h->anchors.front();
-        h->anchors.pop_front();
+    }
+    if (mirrored->demoted_frame >= 0) {
+      auto it = std::find(h->anchors.begin(), h->anchors.end(), mirrored->demoted_frame);
+      if (it != h->anchors.end()) {
+        h->decided_demote = mirrored->demoted_frame;
+        h->anchors.erase(it);
       }
     }
+  } else if (t != h->first_frame && c.anchor_tokens > 0 && c.k_max > 0 && io->conf != nullptr && io->rho < c.tau &&
+             t - h->last_registration >= c.min_anchor_interval) {
+    h->decided_register = true;
+    h->anchors.push_back(t);
+    h->last_registration = t;
+    if ((int)h->anchors.size() > c.k_max) {
+      h->decided_demote = h->anchors.front();
+      h->anchors.pop_front();
+    }
   }
-  const int per_anchor = c.camera_head ? 1 : c.anchor_tokens;
-  const bool first = (t == h->first_frame);
-  h->last_stream = st_move;
+}
 
-  const bool prelaunched = S.scores_frame == t;    // ovggt_layer_step already enqueued them on st_sel
-  S.scores_frame = -1;
-  if (!prelaunched) {
-    rc = enqueue_scores(h, S, io, st_sel);
-    if (rc) return rc;
-  }
+// Parameter block of the fused selection kernel for the layer's pending frame.
+CompressParams select_params(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io) {
+  const ovggt_config& c = h->cfg;
+  const int b = S.cur;
+  const bool first = io->frame_id == h->first_frame;
   CompressParams P;
-  P.n = n; P.M = M; P.B = B;
+  P.n = S.n; P.M = h->M; P.B = S.budget;
   P.n_special = c.n_special; P.grid_h = c.grid_h; P.grid_w = c.grid_w;
   P.alpha = c.alpha; P.w_center = h->w_center; P.w_edge = h->w_edge; P.w_corner = h->w_corner;
   P.beta = c.beta;
@@ -752,6 +761,7 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
   P.protect_new = (first && c.protect_first_frame) ? OVGGT_FLAG_INIT
                                                    : ((c.camera_head && h->decided_register) ? OVGGT_FLAG_HIST : 0);
   P.lone_new = c.camera_head ? 1.0f : -1.0f;
+  P.step_key = splitmix64(c.random_seed ^ (unsigned long long)io->frame_id);
   P.register_anchor = (!c.camera_head && h->decided_register) ? 1 : 0;
   P.A = c.anchor_tokens;
   P.demote_frame = h->decided_demote;
@@ -760,9 +770,61 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
   P.ids_dst = S.ids[b ^ 1]; P.flags_dst = S.flags[b ^ 1]; P.stored_dst = S.stored[b ^ 1];
   P.r_out = S.r; P.survivors = S.surv;
   P.status = h->status; P.n_keep_out = S.n_keep_dev;
-  P.fill = fill ? 1 : 0;
+  P.fill = fill_layout(h) ? 1 : 0;
   P.slot_src = S.slot[b]; P.slot_dst = S.slot[b ^ 1];
   P.move_src = S.move_src; P.move_dst = S.move_dst; P.move_j = S.move_j; P.n_moves_out = S.n_moves_dev;
+  return P;
+}
+
+// Host bookkeeping that follows deterministically from the sizes once a layer's compress has been enqueued.
+void close_compress(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io) {
+  const ovggt_config& c = h->cfg;
+  const int N = S.n + h->M, n_keep = std::min(N, S.budget);
+  const int per_anchor = c.camera_head ? 1 : c.anchor_tokens;
+  if (io->frame_id == h->first_frame && c.protect_first_frame) S.n_prot_init = h->M;
+  if (h->decided_register) S.n_prot_hist += per_anchor;
+  if (h->decided_demote >= 0) S.n_prot_hist -= per_anchor;
+  S.evicted_total += N - n_keep;
+  S.last_N = N;
+  S.last_keep = n_keep;
+  S.n = n_keep;
+  S.cur ^= 1;
+  S.pending = false;
+  S.frames_seen += 1;
+}
+
+// Does the hole-filling move of this step also leave corrections of the key column sums?  They continue the sums the
+// step's diversity launch used and wrote to ksum[kcur ^ 1], and describe the next cache only if every slot below B
+// held a cached row (n == B: steady state).
+bool move_leaves_corrections(const ovggt_cache* h, const LayerState& S) {
+  return h->cfg.score_mode == OVGGT_SCORE_HYBRID && h->C * h->elem / 16 <= kCompactSumMaxVec && S.n == S.budget;
+}
+
+// The compress half.  Scores and selection go to st_sel.  What moves K/V rows goes to st_move: the stable gather
+// writes another buffer and may run beside an attention that still reads this one (st_move = st_sel); the
+// hole-filling move writes the buffer the attention reads, so it follows both (st_move = the attention's stream,
+// which first waits for st_sel).
+int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st_sel, cudaStream_t st_move,
+                  const MirroredDecision* mirrored = nullptr) {
+  int rc = validate_compress(h, layer, io, mirrored);
+  if (rc) return rc;
+  LayerState& S = h->layers[layer];
+  const ovggt_config& c = h->cfg;
+  const int M = h->M, C = h->C, n = S.n, N = n + M, B = S.budget, b = S.cur, kb = S.kv;
+  const int64_t t = io->frame_id;
+  const bool fill = fill_layout(h);
+  take_decision(h, io, mirrored);     // nothing below can fail on an argument any more
+  h->last_stream = st_move;
+
+  const bool prelaunched = S.scores_frame == t;    // ovggt_layer_step already enqueued them on st_sel
+  S.scores_frame = -1;
+  if (!prelaunched) {
+    rc = enqueue_scores(h, S, io, st_sel);
+    if (rc) return rc;
+  }
+  const CompressParams P = select_params(h, S, io);
+  const int ncta = select_cluster_ctas(N);
+  const size_t smem = compress_smem_bytes((N + ncta - 1) / ncta, h->Np, M);
   CK(cudaFuncSetAttribute(k_compress_select, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit));
   {
     ProfScope ps(h, OVGGT_PROF_SELECT, st_sel);
@@ -770,7 +832,6 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
     LAUNCHED();
   }
   const int n_keep = std::min(N, B);
-  const bool sums_fit = C * h->elem / 16 <= kCompactSumMaxVec;
   if (fill) {
     S.ksum_valid = false;
     if (N > B) {   // some rows leave: survivors above slot B move into the slots that open below it
@@ -778,9 +839,7 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
         CK(cudaEventRecord(h->ev_join, st_sel));
         CK(cudaStreamWaitEvent(st_move, h->ev_join, 0));
       }
-      // The corrections continue the sums this step's diversity launch used and wrote to ksum[kcur ^ 1]; they
-      // describe the next cache only if every slot below B held a cached row (n == B: steady state).
-      const bool delta = c.score_mode == OVGGT_SCORE_HYBRID && sums_fit && n == B;
+      const bool delta = move_leaves_corrections(h, S);
       ProfScope ps(h, OVGGT_PROF_COMPACT, st_move);
       rc = launch_fill_holes(S.kbuf[kb], S.vbuf[kb], S.move_src, S.move_dst, S.move_j, S.n_moves_dev, M, C, c.dtype,
                              S.slot[b ^ 1], delta ? S.ksum[S.kcur ^ 1] + C : nullptr, st_move);
@@ -792,7 +851,7 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
     }
   } else {
     ProfScope ps(h, OVGGT_PROF_COMPACT, st_move);
-    const bool fuse = c.score_mode == OVGGT_SCORE_HYBRID && sums_fit;
+    const bool fuse = c.score_mode == OVGGT_SCORE_HYBRID && C * h->elem / 16 <= kCompactSumMaxVec;
     S.colsum_nparts = 0;
     if (fuse)
       rc = launch_compact_colsum(S.kbuf[kb], S.vbuf[kb], S.surv, n_keep, C, c.dtype, S.kbuf[kb ^ 1], S.vbuf[kb ^ 1],
@@ -802,18 +861,117 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
     if (rc) return rc;
     S.kv = kb ^ 1;
   }
+  close_compress(h, S, io);
+  return OVGGT_OK;
+}
 
-  // bookkeeping that follows deterministically from the sizes
-  if (first && c.protect_first_frame) S.n_prot_init = M;
-  if (h->decided_register) S.n_prot_hist += per_anchor;
-  if (h->decided_demote >= 0) S.n_prot_hist -= per_anchor;
-  S.evicted_total += N - n_keep;
-  S.last_N = N;
-  S.last_keep = n_keep;
-  S.n = n_keep;
-  S.cur = b ^ 1;
-  S.pending = false;
-  S.frames_seen += 1;
+// The compress half of every layer of the handle for one frame, in three launches instead of three per layer
+// (hole-filling layout; the batched kernels take one parameter block per layer as kernel arguments).
+int compress_all_layers(ovggt_cache* h, const ovggt_frame_io* ios, cudaStream_t st) {
+  const ovggt_config& c = h->cfg;
+  const int L = (int)h->layers.size(), M = h->M, C = h->C;
+  for (int l = 0; l < L; ++l) {
+    int rc = validate_compress(h, l, &ios[l], nullptr);
+    if (rc) return rc;
+    if (ios[l].frame_id != ios[0].frame_id) return OVGGT_ERR_FRAME_ORDER;
+  }
+  if (!fill_layout(h)) {                     // the stable gather has no batched kernels: layer by layer
+    for (int l = 0; l < L; ++l) {
+      int rc = compress_impl(h, l, &ios[l], st, st);
+      if (rc) return rc;
+    }
+    return OVGGT_OK;
+  }
+  take_decision(h, &ios[0], nullptr);
+  h->last_stream = st;
+  const int nvec = C * h->elem / 16;
+  CK(cudaFuncSetAttribute(k_compress_select_batched, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit));
+  for (int l0 = 0; l0 < L; l0 += kMaxBatchLayers) {
+    const int cnt = std::min(kMaxBatchLayers, L - l0);
+    // ---- scores: diversity of the cached keys and the frame's residual norms
+    {
+      ProfScope ps(h, OVGGT_PROF_DIVERSITY, st);
+      DiversityBatch db;
+      int grid_x = 1;
+      for (int i = 0; i < cnt; ++i) {
+        LayerState& S = h->layers[l0 + i];
+        S.scores_frame = -1;
+        const bool hybrid = c.score_mode == OVGGT_SCORE_HYBRID && S.n > 0;
+        DiversityArgs& A = db.a[i];
+        A = DiversityArgs{};
+        A.resid = (const uint4*)ios[l0 + i].resid; A.resid_rows = M; A.s_raw = S.s_raw;
+        if (hybrid) {
+          const bool fresh = !S.ksum_valid || S.since_refresh >= kColsumRefreshEvery;
+          if (fresh) {
+            int rc = launch_colsum(S.kbuf[S.kv], S.n, C, c.dtype, h->colsum_part, S.ksum[S.kcur], st);
+            if (rc) return rc;
+            S.since_refresh = 0;
+          } else {
+            S.since_refresh += 1;
+          }
+          A.K = (const uint4*)S.kbuf[S.kv]; A.rows = S.n;
+          A.ksum = S.ksum[S.kcur]; A.n_slices = fresh ? 1 : 1 + kFillSlices; A.ksum_out = S.ksum[S.kcur ^ 1];
+          A.d = S.d;
+          A.div_ctas = std::min((S.n + 63) / 64, 148 * 8);
+        }
+        grid_x = std::max(grid_x, A.div_ctas + (M + 7) / 8);
+      }
+      if (c.dtype == kBF16) k_diversity_batched<kBF16><<<dim3(grid_x, cnt), 256, (size_t)C * 4, st>>>(db, nvec);
+      else                  k_diversity_batched<kF32><<<dim3(grid_x, cnt), 256, (size_t)C * 4, st>>>(db, nvec);
+      LAUNCHED();
+    }
+    // ---- flags, Eq. 6-8, compacted meta, move pairs: one cluster per layer
+    {
+      ProfScope ps(h, OVGGT_PROF_SELECT, st);
+      CompressBatch cb;
+      int n_max = 0;
+      for (int i = 0; i < cnt; ++i) {
+        LayerState& S = h->layers[l0 + i];
+        cb.p[i] = select_params(h, S, &ios[l0 + i]);
+        n_max = std::max(n_max, S.n + M);
+      }
+      const int ncta = select_cluster_ctas(n_max);
+      const size_t smem = compress_smem_bytes((n_max + ncta - 1) / ncta, h->Np, M);
+      CK(launch_cluster(k_compress_select_batched, dim3(ncta, cnt), ncta, smem, st, cb));
+      LAUNCHED();
+    }
+    // ---- the moves of the layers that evict
+    {
+      ProfScope ps(h, OVGGT_PROF_COMPACT, st);
+      FillBatch fb;
+      int nf = 0;
+      for (int i = 0; i < cnt; ++i) {
+        LayerState& S = h->layers[l0 + i];
+        S.ksum_valid = false;
+        if (S.n + M <= S.budget) continue;
+        const bool delta = move_leaves_corrections(h, S);
+        fb.a[nf++] = FillArgs{(uint4*)S.kbuf[S.kv], (uint4*)S.vbuf[S.kv], S.move_src, S.move_dst, S.move_j, S.n_moves_dev,
+                              M, S.slot[S.cur ^ 1], delta ? S.ksum[S.kcur ^ 1] + C : nullptr};
+        if (delta) {
+          S.kcur ^= 1;
+          S.ksum_valid = true;
+        }
+      }
+      if (nf > 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kFillSlices * kFillClusterCtas, nf);
+        cfg.blockDim = dim3(kFillThreads);
+        cfg.stream = st;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = kFillClusterCtas;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = c.dtype == kBF16 ? cudaLaunchKernelEx(&cfg, k_fill_holes_batched<kBF16>, fb, nvec)
+                                         : cudaLaunchKernelEx(&cfg, k_fill_holes_batched<kF32>, fb, nvec);
+        if (e != cudaSuccess) return cuda_fail(e);
+        LAUNCHED();
+      }
+    }
+    for (int i = 0; i < cnt; ++i) close_compress(h, h->layers[l0 + i], &ios[l0 + i]);
+  }
   return OVGGT_OK;
 }
 }  // namespace
@@ -845,6 +1003,11 @@ extern "C" int ovggt_camera_compress(ovggt_cache* h, int32_t layer, const ovggt_
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const MirroredDecision d{registered != 0, demoted_frame};
   return compress_impl(h, layer, io, st, st, &d);
+}
+
+extern "C" int ovggt_layers_compress(ovggt_cache* h, const ovggt_frame_io* ios, int32_t n_ios, void* stream) {
+  if (!h || !ios || n_ios != (int32_t)h->layers.size() || h->cfg.camera_head) return OVGGT_ERR_INVALID_ARG;
+  return compress_all_layers(h, ios, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
@@ -888,6 +1051,12 @@ extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame
   if (rc) return rc;
   if (e1 != cudaSuccess) return cuda_fail(e1);
   if (e2 != cudaSuccess) return cuda_fail(e2);
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_cache_set_key_bound(ovggt_cache* h, int32_t enable) {
+  if (!h) return OVGGT_ERR_INVALID_ARG;
+  h->use_key_bound = enable != 0;
   return OVGGT_OK;
 }
 
@@ -1064,6 +1233,12 @@ extern "C" int ovggt_cache_import(ovggt_cache* h, int32_t layer, const int64_t* 
       CK(cudaMemcpy(S.slot[b], slot.data(), (size_t)n * 4, cudaMemcpyHostToDevice));
     }
   }
+  CK(cudaMemset(S.kmax2, 0, (size_t)h->cfg.n_heads * 4));
+  if (n > 0 && h->cfg.dtype == kBF16 && h->C * h->elem / 16 <= 128) {
+    k_key_norm_max<<<std::min((n + 7) / 8, 148 * 8), 256>>>((const uint4*)S.kbuf[kb], n, h->C * h->elem / 16, S.kmax2);
+    LAUNCHED();
+    CK(cudaDeviceSynchronize());
+  }
   S.n = n;
   S.colsum_nparts = 0;          // the imported keys have not been summed
   S.ksum_valid = false;
@@ -1097,6 +1272,7 @@ extern "C" int ovggt_cache_reset(ovggt_cache* h) {
     S.ksum_valid = false;
     S.since_refresh = 0;
     S.scores_frame = -1;
+    CK(cudaMemset(S.kmax2, 0, (size_t)h->cfg.n_heads * 4));
   }
   h->anchors.clear();
   h->first_frame = h->last_registration = h->decided_frame = -1;
@@ -1254,6 +1430,27 @@ extern "C" int ovggt_k_attention(const void* q, const void* k, const void* v, in
   if (dtype == kBF16 && (!scratch || !device_status)) return OVGGT_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return OVGGT_ERR_MISALIGNED;
   return launch_attention(q, k, v, M, N, n_heads, dtype, out, scratch, device_status, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int ovggt_k_key_norm_bound(const void* K, int32_t rows, int32_t n_heads, float* kmax2, void* stream) {
+  if (!kmax2 || rows < 0 || (rows > 0 && !K) || n_heads < 1 || n_heads > 16) return OVGGT_ERR_INVALID_ARG;
+  if (!aligned16(K)) return OVGGT_ERR_MISALIGNED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CK(cudaMemsetAsync(kmax2, 0, (size_t)n_heads * 4, st));
+  if (rows == 0) return OVGGT_OK;
+  k_key_norm_max<<<std::min((rows + 7) / 8, 148 * 8), 256, 0, st>>>((const uint4*)K, rows, n_heads * 8, kmax2);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
+extern "C" int ovggt_k_attention_bounded(const void* q, const void* k, const void* v, int32_t M, int32_t N,
+                                         int32_t n_heads, void* out, void* scratch, int32_t* device_status,
+                                         const float* kmax2, void* stream) {
+  if (!q || !k || !v || !out || M < 1 || N < 1 || n_heads < 1 || !scratch || !device_status || !kmax2)
+    return OVGGT_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return OVGGT_ERR_MISALIGNED;
+  return launch_attention(q, k, v, M, N, n_heads, kBF16, out, scratch, device_status, static_cast<cudaStream_t>(stream),
+                          nullptr, kmax2);
 }
 
 // ------------------------------------------------------------------ allocation-free diversity

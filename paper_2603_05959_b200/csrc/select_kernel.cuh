@@ -278,6 +278,7 @@ struct CompressParams {
   float beta;
   int mode;                         // OVGGT_SCORE_*
   int protect_new;                  // != 0: give every new row this flag (INIT: first frame; HIST: a camera-cache anchor)
+  unsigned long long step_key;      // OVGGT_SCORE_RANDOM: SplitMix64(seed ^ frame id) of this step
   float lone_new;                   // >= 0: normalised score of a new group without a range (Eq. 7's 0/0); < 0: 0
   int register_anchor, A;           // 1: flag the A most confident patches of the new frame HIST
   long long demote_frame;           // >= 0: release the HIST rows of that frame
@@ -402,6 +403,7 @@ __device__ __forceinline__ void compress_select_body(const CompressParams& P, un
           x = (P.mode == OVGGT_SCORE_HYBRID) ? d4[u] : st4[u];
           keepscore = st4[u];
         }
+        if (P.mode == OVGGT_SCORE_RANDOM) x = random_priority(P.step_key, id4[u]);   // Supp. A: uniform, fresh per step
         fl[i] = f;
         val[i] = x;
         sid[i] = id4[u];

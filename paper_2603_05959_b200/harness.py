@@ -162,9 +162,13 @@ class Aggregator:
     global-attention block (the library: attention over the bounded cache), each followed by an MLP of width 4C,
     random-init N(0, 0.02), LayerScale taken as 1.  In the global block the library's two halves bracket the MLP:
     attend -> h = x + O W_o -> r = MLP(LN(h)) -> compress(resid = r) -> x = h + r, so the activation score sees the
-    block's real MLP output.  `tap` and `after` as in ProjectionStack."""
+    block's real MLP output.  With batched_compress the compress of all layers is deferred to the end of the frame and
+    issued as one call (ovggt_layers_compress): that is the order a real model needs, whose anchor inputs (coverage,
+    confidence) come out of its heads after the last block.  `tap` and `after` as in ProjectionStack."""
 
-    def __init__(self, cfg: gen.StreamConfig, device, compaction: int = B.COMPACT_FILL_HOLES):
+    def __init__(self, cfg: gen.StreamConfig, device, compaction: int = B.COMPACT_FILL_HOLES,
+                 batched_compress: bool = True):
+        self.batched_compress = batched_compress
         assert cfg.dtype == gen.DTYPE_BF16
         self.cfg, self.device = cfg, device
         self.cache = B.OvggtCache.from_stream(cfg, device=device, compaction=compaction)
@@ -185,6 +189,7 @@ class Aggregator:
               lib: Optional[_Timer] = None) -> torch.Tensor:
         cfg = self.cfg
         C, H, M = cfg.dim, cfg.n_heads, cfg.tokens_per_frame
+        resids, overrides = [], []
         for l in range(cfg.n_layers):
             w = self.blocks[l]["frame"]
             qkv = (_layer_norm(x) @ w["qkv"]).view(M, 3, H, C // H).permute(1, 2, 0, 3)        # [3, H, M, d]
@@ -201,9 +206,17 @@ class Aggregator:
             h = x + self.out @ w["o"]
             r = self._mlp(w, h).contiguous()
             ov = self.tap(t, l, q, k, v, r) if self.tap else None
-            cmp_ = lambda: self.cache.layer_compress(l, t, r, conf, rho, score_override=ov, stream=stream)
-            lib(cmp_) if lib else cmp_()
+            if self.batched_compress:
+                resids.append(r)
+                overrides.append(ov)
+            else:
+                cmp_ = lambda: self.cache.layer_compress(l, t, r, conf, rho, score_override=ov, stream=stream)
+                lib(cmp_) if lib else cmp_()
             x = h + r
+        if self.batched_compress:
+            ovs = overrides if any(o is not None for o in overrides) else None
+            cmp_ = lambda: self.cache.layers_compress(t, resids, conf, rho, score_overrides=ovs, stream=stream)
+            lib(cmp_) if lib else cmp_()
         return x
 
     def destroy(self) -> None:

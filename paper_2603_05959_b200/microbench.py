@@ -74,11 +74,19 @@ def bench_attention(args):
     out = torch.empty_like(q)
     scratch = torch.empty(B.lib().ovggt_k_attention_scratch_bytes(M, N, H), dtype=torch.uint8, device="cuda")
     status = torch.zeros(16, dtype=torch.int32, device="cuda")
-    fn = lambda: B.k_attention(q, k, v, H, out=out, scratch=scratch, status=status)
+    if args.tracked_max:
+        fn = lambda: B.k_attention(q, k, v, H, out=out, scratch=scratch, status=status)
+    else:
+        # the library's own call: the key-norm bound exists before the attention runs (the append keeps it)
+        kmax2 = B.k_key_norm_bound(k, H)
+        sp = torch.cuda.current_stream().cuda_stream
+        fn = lambda: B.lib().ovggt_k_attention_bounded(q.data_ptr(), k.data_ptr(), v.data_ptr(), M, N, H, out.data_ptr(),
+                                                       scratch.data_ptr(), status.data_ptr(), kmax2.data_ptr(), sp)
     ms = Timer(args.flush).run(fn, args.iters)
     assert int(status[0].item()) == 0
     return _emit("attention (k_attn_tcgen05 + k_attn_merge)", ms, {"M": M, "N": N, "heads": H},
-                 flops=4.0 * M * N * C, extra={"kv_mb": 4 * N * C / 1e6})
+                 flops=4.0 * M * N * C, extra={"kv_mb": 4 * N * C / 1e6,
+                                               "softmax_reference": "tracked maximum" if args.tracked_max else "key-norm bound"})
 
 
 def bench_row_norms(args):
@@ -127,6 +135,7 @@ def main():
     ap.add_argument("--batch", type=int, default=64)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--flush", action="store_true", help="write a 252 MB buffer between iterations")
+    ap.add_argument("--tracked-max", action="store_true", help="attention without the key-norm bound")
     args = ap.parse_args()
     torch.cuda.set_device(0)
     todo = ["attention", "row_norms", "diversity", "select", "compact"] if args.kernel == "all" else [args.kernel]

@@ -39,13 +39,13 @@ def test_library_exports_every_declared_symbol(lib):
 def _cfg(**over):
     kw = dict(n_layers=1, n_heads=4, head_dim=64, n_special=5, grid_h=8, grid_w=8, budget=256,
               anchor_tokens=8, k_max=3, min_anchor_interval=4, tau=0.2, alpha=0.5, beta=0.5,
-              protect_first_frame=1, score_mode=0, dtype=0, compaction=1, camera_head=0)
+              protect_first_frame=1, score_mode=0, dtype=0, compaction=1, random_seed=0, camera_head=0)
     kw.update(over)
     budgets = (C.c_int32 * kw["n_layers"])(*([kw.pop("budget")] * kw["n_layers"]))
     cfg = B.OvggtConfig(kw["n_layers"], kw["n_heads"], kw["head_dim"], kw["n_special"], kw["grid_h"],
                         kw["grid_w"], budgets, kw["anchor_tokens"], kw["k_max"], kw["min_anchor_interval"],
                         kw["tau"], kw["alpha"], kw["beta"], kw["protect_first_frame"], kw["score_mode"],
-                        kw["dtype"], kw["compaction"], kw["camera_head"], None, 0)
+                        kw["dtype"], kw["compaction"], kw["random_seed"], kw["camera_head"], None, 0)
     cfg._keep = budgets
     return cfg
 
@@ -68,7 +68,7 @@ def test_workspace_bytes_is_a_pure_host_function(lib):
 def test_create_reports_config_errors_without_a_gpu(lib):
     h = C.c_void_p()
     bad = [(_cfg(head_dim=32), -1), (_cfg(n_layers=0, budget=256), -1), (_cfg(dtype=7), -1),
-           (_cfg(alpha=1.5), -1), (_cfg(k_max=17), -1), (_cfg(anchor_tokens=65), -1), (_cfg(compaction=2), -1),
+           (_cfg(alpha=1.5), -1), (_cfg(k_max=17), -1), (_cfg(anchor_tokens=65), -1), (_cfg(compaction=2), -1), (_cfg(score_mode=3), -1),
            (_cfg(camera_head=1), -1), (_cfg(camera_head=1, n_special=1, grid_h=0, grid_w=0, anchor_tokens=0, budget=3), -3),
            (_cfg(budget=68), -3), (_cfg(budget=69 + 3 * 8 - 1), -3)]
     for cfg, code in bad:

@@ -146,13 +146,14 @@ def test_projection_stack_harness_library_calls_match_the_oracle():
     model.destroy()
 
 
-def test_aggregator_harness_library_calls_match_the_oracle():
+@pytest.mark.parametrize("batched", [True, False], ids=["compress-all-layers-at-frame-end", "compress-per-layer"])
+def test_aggregator_harness_library_calls_match_the_oracle(batched):
     """The alternating-aggregator harness (frame attention and MLPs in torch; attend -> MLP -> compress around the
     library, the activation score fed by the block's real MLP output), cut to 2 depths: every library call against
     the oracle, on the 1041-token layout."""
     from paper_2603_05959_b200 import harness as H
     cfg = gen.config_aggregator().replace(n_layers=2, budget=2500, min_anchor_interval=2, tau=0.8)
-    model = H.Aggregator(cfg, torch.device("cuda", torch.cuda.current_device()))
+    model = H.Aggregator(cfg, torch.device("cuda", torch.cuda.current_device()), batched_compress=batched)
     stream = torch.cuda.current_stream()
     rows = np.array([0, 3, 5, 512, 1040], dtype=np.int32)
 

@@ -106,9 +106,12 @@ def test_compact_is_exact_gather(C, dtype):
     assert kd.shape[0] == 0
 
 
-def _attn_check(M, N, H, dtype, seed, rows=None, qscale=1.0):
+BOTH_REFERENCES = pytest.mark.parametrize("bounded", [False, True], ids=["tracked-max", "key-bound"])
+
+
+def _attn_check(M, N, H, dtype, seed, rows=None, qscale=1.0, bounded=False):
     q, k, v = rnd((M, H * 64), dtype, seed, qscale), rnd((N, H * 64), dtype, seed + 1), rnd((N, H * 64), dtype, seed + 2)
-    got = B.k_attention(dev(q, dtype), dev(k, dtype), dev(v, dtype), H).float().cpu().numpy()
+    got = B.k_attention(dev(q, dtype), dev(k, dtype), dev(v, dtype), H, bounded=bounded).float().cpu().numpy()
     assert np.isfinite(got).all()
     ref = orc.attention(q, k, v, H, 64, rows=rows)
     g = got if rows is None else got[rows]
@@ -122,19 +125,33 @@ def _attn_check(M, N, H, dtype, seed, rows=None, qscale=1.0):
 
 @pytest.mark.parametrize("M,N,H", [(128, 128, 1), (1, 1, 1), (94, 129, 2), (200, 1000, 2), (69, 325, 4),
                                    (300, 4096, 3), (129, 2500, 1)])
-def test_attention_bf16_small(M, N, H):
+@BOTH_REFERENCES
+def test_attention_bf16_small(M, N, H, bounded):
     orc.set_threads(8)
-    _attn_check(M, N, H, gen.DTYPE_BF16, 10 + M + N)
+    _attn_check(M, N, H, gen.DTYPE_BF16, 10 + M + N, bounded=bounded)
 
 
-def test_attention_bf16_large_logits_exercise_rescaling():
+@BOTH_REFERENCES
+def test_attention_bf16_large_logits_exercise_rescaling(bounded):
     orc.set_threads(8)
-    _attn_check(150, 1500, 2, gen.DTYPE_BF16, 77, qscale=6.0)
+    _attn_check(150, 1500, 2, gen.DTYPE_BF16, 77, qscale=6.0, bounded=bounded)
 
 
-def test_attention_bf16_scores_rising_along_the_keys():
+def test_key_norm_bound_is_the_largest_per_head_key_norm():
+    k = rnd((3001, 5 * 64), gen.DTYPE_BF16, 3) * np.linspace(0.5, 2.0, 5, dtype=np.float32).repeat(64)[None, :]
+    k = gen.round_to_dtype(k, gen.DTYPE_BF16)
+    got = B.k_key_norm_bound(dev(k, 1), 5).cpu().numpy()
+    want = (k.astype(np.float64).reshape(3001, 5, 64) ** 2).sum(-1).max(0)
+    np.testing.assert_allclose(got, want, rtol=1e-5)
+    assert B.k_key_norm_bound(torch.empty((0, 128), dtype=torch.bfloat16, device="cuda"), 2).tolist() == [0.0, 0.0]
+
+
+@BOTH_REFERENCES
+def test_attention_bf16_scores_rising_along_the_keys(bounded):
     """Keys ordered so that every score half outgrows the running reference maximum by far more than the lazy
-    threshold: each round takes the rescale-and-recompute path, and the softmax concentrates on the last keys."""
+    threshold: each round takes the rescale-and-recompute path, and the softmax concentrates on the last keys.
+    (With the key-norm bound on, that bound lies hundreds of powers of two above the first scores, which the kernel
+    must notice and fall back to tracking the maximum.)"""
     orc.set_threads(8)
     M, N, H, dt = 140, 1100, 2, gen.DTYPE_BF16
     rng = np.random.default_rng(91)
@@ -145,7 +162,7 @@ def test_attention_bf16_scores_rising_along_the_keys():
     q = np.concatenate([(8.0 + rng.random((M, 1)).astype(np.float32)) * u[None, :] for _ in range(H)], axis=1)
     v = rng.standard_normal((N, H * 64)).astype(np.float32)
     q, k, v = (gen.round_to_dtype(x, dt) for x in (q, k, v))
-    got = B.k_attention(dev(q, dt), dev(k, dt), dev(v, dt), H).float().cpu().numpy()
+    got = B.k_attention(dev(q, dt), dev(k, dt), dev(v, dt), H, bounded=bounded).float().cpu().numpy()
     ref = orc.attention(q, k, v, H, 64)
     err = np.abs(got - ref)
     assert np.isfinite(got).all() and err.max() <= ATT_MAX and err.mean() <= ATT_MEAN, (err.max(), err.mean())
@@ -157,17 +174,19 @@ def test_attention_fp32(M, N, H):
     _attn_check(M, N, H, gen.DTYPE_F32, 20 + M)
 
 
-def test_attention_bf16_full_size_sampled_rows():
+@BOTH_REFERENCES
+def test_attention_bf16_full_size_sampled_rows(bounded):
     """The bench configuration: 1374 queries x 17758 keys x 16 heads; the oracle checks sampled rows."""
     orc.set_threads(max(1, min(32, torch.get_num_threads())))
     rows = np.sort(np.random.default_rng(5).choice(1374, 24, replace=False)).astype(np.int32)
     rows[0], rows[-1] = 0, 1373
-    got = _attn_check(1374, 17758, 16, gen.DTYPE_BF16, 30, rows=rows)
+    got = _attn_check(1374, 17758, 16, gen.DTYPE_BF16, 30, rows=rows, bounded=bounded)
     # properties that hold at any size: finite, and each output inside the range of V per column
     assert np.abs(got).max() < 6.0
 
 
-def test_attention_bf16_full_size_peaked_logits_every_key_block_matters():
+@BOTH_REFERENCES
+def test_attention_bf16_full_size_peaked_logits_every_key_block_matters(bounded):
     """The bench shape again (5 KV splits x 19 tiles, 94-row tail, ragged last query tile) on data that can fail it:
     see tiled_hot_case.  As a self-check of the data, the reference is recomputed without the last key block and
     without the middle fifth of the keys and must then violate the criterion the kernel has to meet."""
@@ -176,7 +195,7 @@ def test_attention_bf16_full_size_peaked_logits_every_key_block_matters():
     q, k, v = tiled_hot_case(M, N, H, 41)
     rows = sampled_rows_all_groups(M)
     assert len(rows) >= 24 and rows.max() >= 1280
-    got = B.k_attention(dev(q, 1), dev(k, 1), dev(v, 1), H).float().cpu().numpy()
+    got = B.k_attention(dev(q, 1), dev(k, 1), dev(v, 1), H, bounded=bounded).float().cpu().numpy()
     assert np.isfinite(got).all()
     ref = orc.attention(q, k, v, H, 64, rows=rows)
     assert_attention_close_relative(got[rows], ref, "bench shape, peaked")
@@ -187,12 +206,13 @@ def test_attention_bf16_full_size_peaked_logits_every_key_block_matters():
             assert_attention_close_relative(broken, ref)
 
 
+@BOTH_REFERENCES
 @pytest.mark.parametrize("M,N,H", [(300, 2500, 2), (1041, 13329, 2)])
-def test_attention_bf16_peaked_logits_other_shapes(M, N, H):
+def test_attention_bf16_peaked_logits_other_shapes(M, N, H, bounded):
     orc.set_threads(max(1, min(32, torch.get_num_threads())))
     q, k, v = tiled_hot_case(M, N, H, 43 + M)
     rows = sampled_rows_all_groups(M)
-    got = B.k_attention(dev(q, 1), dev(k, 1), dev(v, 1), H).float().cpu().numpy()
+    got = B.k_attention(dev(q, 1), dev(k, 1), dev(v, 1), H, bounded=bounded).float().cpu().numpy()
     assert_attention_close_relative(got[rows], orc.attention(q, k, v, H, 64, rows=rows), f"{M}x{N}")
 
 

@@ -103,6 +103,31 @@ def test_stored_residual_mode_and_no_anchors():
     run_teacher_forced(cfg, 8, attn_frames={7})
 
 
+def test_random_eviction_mode_runs_free_and_matches_the_oracle_bit_for_bit():
+    """The random-eviction baseline (Supp. A).  Its priorities are counter-based values that both sides compute
+    from (seed, frame, token id) exactly, so no teacher forcing is needed: the library runs freely and must keep the
+    oracle's survivors, priorities and layout bit for bit, in both layouts."""
+    cfg = gen.StreamConfig(name="rnd", n_heads=2, grid_h=7, grid_w=9, budget=250, anchor_tokens=5, k_max=2,
+                           min_anchor_interval=3, tau=0.9, n_frames=25, dtype=gen.DTYPE_F32, score_mode=gen.SCORE_RANDOM)
+    for compaction in (B.COMPACT_FILL_HOLES, B.COMPACT_STABLE_GATHER):
+        layer = orc.OracleLayer.from_stream(cfg)
+        c = B.OvggtCache.from_stream(cfg, compaction=compaction)
+        for t in range(cfg.n_frames):
+            fi = gen.frame_inputs(cfg, t)
+            df = DeviceFrame(cfg, fi, "cuda")
+            layer.attend(t, fi.q, fi.k, fi.v, compute=False)
+            ref = layer.compress(fi.resid, fi.conf, fi.rho)
+            c.layer_step(0, t, df.q, df.k, df.v, df.resid, df.conf, df.rho)
+            sel = c.last_selection(0)
+            np.testing.assert_array_equal(sel["survivors"], ref["survivors"], err_msg=f"frame {t}")
+            np.testing.assert_array_equal(sel["r"], ref["r"], err_msg=f"frame {t}")
+        ex, rx = c.export(0), layer.export()
+        np.testing.assert_array_equal(ex["ids"], rx["ids"])
+        np.testing.assert_array_equal(ex["flags"], rx["flags"])
+        assert np.array_equal(ex["k"], rx["k"]) and layer.evicted_total > 0
+        c.destroy()
+
+
 @BOTH_LAYOUTS
 def test_bf16_ragged_midsize_stream(compaction):
     """Several KV tiles with a ragged tail, two ragged query tiles, bf16, anchors on."""
@@ -367,6 +392,55 @@ def test_config2_full_size_stream_teacher_forced(compaction):
     threads = max(1, min(32, torch.get_num_threads()))
     run_teacher_forced(cfg, 40, attn_frames={0, 11, 12, 39}, attn_rows=rows, export_every=13, threads=threads,
                        compaction=compaction)
+
+
+@pytest.mark.parametrize("dtype,compaction", [(gen.DTYPE_F32, B.COMPACT_FILL_HOLES), (gen.DTYPE_BF16, B.COMPACT_FILL_HOLES),
+                                              (gen.DTYPE_F32, B.COMPACT_STABLE_GATHER)])
+def test_all_layers_compressed_in_one_call_with_per_layer_budgets(dtype, compaction):
+    """ovggt_layers_compress: three layers with budgets of their own (Sec. 3.2), attended one by one and compressed
+    together - the way a model works whose anchor inputs exist only after its heads.  Teacher-forced per layer, so
+    survivors, priorities, counters and exported layouts must match three independent oracles frame by frame."""
+    budgets = [256, 150, 333]
+    cfg = gen.config_tiny().replace(n_layers=3, tau=0.9, min_anchor_interval=2, k_max=2, n_frames=14, dtype=dtype)
+    c = B.OvggtCache.from_stream(cfg, budget=budgets, compaction=compaction)
+    oracles = [orc.OracleLayer.from_stream(cfg.replace(budget=b)) for b in budgets]
+    orc.set_threads(4)
+    for t in range(cfg.n_frames):
+        frames, refs, outs, ref_outs = [], [], [], []
+        for l in range(3):
+            fi = gen.frame_inputs(cfg, t, layer=l)
+            df = DeviceFrame(cfg, fi, "cuda")
+            frames.append(df)
+            ref_outs.append(oracles[l].attend(t, fi.q, fi.k, fi.v))
+            refs.append(oracles[l].compress(fi.resid, fi.conf, fi.rho))
+            outs.append(c.layer_attend(l, t, df.q, df.k, df.v))
+        c.layers_compress(t, [f.resid for f in frames], frames[0].conf, frames[0].rho,
+                          score_overrides=[torch.from_numpy(r["r"]).cuda() for r in refs])
+        for l in range(3):
+            err = np.abs(out_to_f32(outs[l]) - ref_outs[l])
+            assert err.max() <= (ATT_F32 if dtype == gen.DTYPE_F32 else ATT_MAX), (t, l, err.max())
+            sel = c.last_selection(l)
+            np.testing.assert_array_equal(sel["survivors"], refs[l]["survivors"], err_msg=f"frame {t} layer {l}")
+            fin = np.isfinite(refs[l]["r"])
+            np.testing.assert_allclose(sel["r"][fin], refs[l]["r"][fin], rtol=0, atol=R_ATOL, err_msg=f"frame {t} layer {l}")
+            st = c.stats(l)
+            assert st["device_status"] == 0 and st["n_cached"] == oracles[l].n_rows == min((t + 1) * cfg.tokens_per_frame, budgets[l])
+            assert st["anchor_frames"] == oracles[l].anchors() and st["evicted_total"] == oracles[l].evicted_total
+            assert (st["n_protected_init"], st["n_protected_hist"]) == oracles[l].protected()
+    for l in range(3):
+        ex, rx = c.export(l), oracles[l].export()
+        np.testing.assert_array_equal(ex["ids"], rx["ids"])
+        np.testing.assert_array_equal(ex["flags"], rx["flags"])
+        np.testing.assert_allclose(ex["stored"], rx["stored"], rtol=STORED_RTOL)
+        assert np.array_equal(storage_to_f32(ex["k"], cfg.dtype), rx["k"])
+        assert np.array_equal(storage_to_f32(ex["v"], cfg.dtype), rx["v"])
+    # the call checks every layer before it changes anything
+    f = frames[0]
+    c.layer_attend(0, cfg.n_frames, f.q, f.k, f.v)           # only layer 0 has a pending frame now
+    with pytest.raises(B.OvggtError) as e:
+        c.layers_compress(cfg.n_frames, [f.resid] * 3, f.conf, f.rho)
+    assert e.value.code == -4 and c.stats(0)["frames_seen"] == cfg.n_frames
+    c.destroy()
 
 
 def test_config2_full_size_through_layer_step_with_overlap():
