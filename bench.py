@@ -425,10 +425,11 @@ def run_c2(args) -> None:
         peak = float(peaks["bf16_tflops"])
         eb = cfg.elem_bytes
         fill = compaction == B.COMPACT_FILL_HOLES
-        alg_bytes = {"append": 4 * M * C * eb, "row_norms": M * C * eb + 4 * M,
+        # hole filling: the append launch also carries the previous step's moves (at most M rows of K and V read and
+        # written again); stable gather: all B rows are read and written by the compaction
+        alg_bytes = {"append": (8 if fill else 4) * M * C * eb, "row_norms": M * C * eb + 4 * M,
                      "diversity": Bud * C * eb + 4 * Bud + M * C * eb + 4 * M, "select": 4 * N + N + 4 * Bud,
-                     # hole filling: the <= M admitted rows are read and written (K and V); stable gather: all B rows
-                     "compact": 4 * min(M, Bud) * C * eb if fill else 4 * Bud * C * eb}
+                     "compact": 4 * Bud * C * eb}
         kernels = kernel_table(prof, alg_bytes, peaks, clocks.get("sm_mhz"))
         if cfg.dtype == gen.DTYPE_BF16:
             kernels["attention"].update({"tflops": achieved, "frac_of_burst_peak": achieved / peak,
@@ -545,9 +546,8 @@ def run_stack(args) -> None:
     achieved = attn_flops / (attn_ms * 1e-3) / 1e12
     peak = float(peaks["bf16_tflops"])
     eb = cfg.elem_bytes
-    alg_bytes = {"append": 4 * M * C * eb, "row_norms": M * C * eb + 4 * M,
-                 "diversity": Bud * C * eb + 4 * Bud + M * C * eb + 4 * M, "select": 4 * N + N + 4 * Bud,
-                 "compact": 4 * M * C * eb}
+    alg_bytes = {"append": 8 * M * C * eb, "row_norms": M * C * eb + 4 * M,
+                 "diversity": Bud * C * eb + 4 * Bud + M * C * eb + 4 * M, "select": 4 * N + N + 4 * Bud}
     line = {"metric": METRIC, "value": K / (total_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W,
             "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",

@@ -13,7 +13,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libovggt.so")
+# OVGGT_LIBRARY=checked selects the build with range-checked indices (paper_2603_05959_b200/build.py --checked)
+LIB_PATH = os.path.join(_HERE, "libovggt_checked.so" if os.environ.get("OVGGT_LIBRARY") == "checked" else "libovggt.so")
 MAX_ANCHORS = 16
 
 DTYPE_F32, DTYPE_BF16 = 0, 1

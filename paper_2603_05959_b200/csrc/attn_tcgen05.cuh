@@ -51,10 +51,13 @@ constexpr float kRescaleThreshold = 8.0f;          // log2 units
 // The price is that every exponential comes out 2^-(bound - true maximum) smaller than it could; fp32 sums and bf16
 // probabilities keep their relative precision as long as that stays far from the underflow threshold (2^-126).
 constexpr float kFixedRefMaxGap = 48.0f;           // log2 units between the bound and the first half's true maximum
-#ifndef OVGGT_ATTN_POLY_EVERY
-#define OVGGT_ATTN_POLY_EVERY 4
+#ifndef OVGGT_ATTN_POLY_NUM
+#define OVGGT_ATTN_POLY_NUM 1
+#define OVGGT_ATTN_POLY_DEN 3
 #endif
-constexpr int kPolyEvery = OVGGT_ATTN_POLY_EVERY;  // one pair of exponentials in kPolyEvery goes to the FMA pipes
+// kPolyNum pairs of exponentials in every kPolyDen go to the FMA pipes instead of the special-function unit
+constexpr int kPolyNum = OVGGT_ATTN_POLY_NUM, kPolyDen = OVGGT_ATTN_POLY_DEN;
+__host__ __device__ constexpr bool pair_on_fma_pipes(int pair) { return (pair * kPolyNum) % kPolyDen < kPolyNum; }
 constexpr int kMaxSplits = 16;
 
 struct AttnBarriers {
@@ -516,7 +519,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           const float s0 = __uint_as_float(s[j]), s1 = __uint_as_float(s[j + 1]);
           if constexpr (decltype(track)::value) m4[(j >> 1) & 3] = max3(m4[(j >> 1) & 3], s0, s1);
           const float2 x = fma2(make_float2(s0, s1), c2, nm2);
-          const float2 p = ((j >> 1) % kPolyEvery == kPolyEvery - 1) ? ex2_poly2(x) : make_float2(ex2(x.x), ex2(x.y));
+          const float2 p = pair_on_fma_pipes(j >> 1) ? ex2_poly2(x) : make_float2(ex2(x.x), ex2(x.y));
           acc[(j >> 1) & 3] = add2(acc[(j >> 1) & 3], p);
           s[j >> 1] = pack_bf16(p.x, p.y);
         }

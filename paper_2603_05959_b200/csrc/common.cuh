@@ -72,6 +72,20 @@ __host__ __device__ __forceinline__ float random_priority(unsigned long long ste
   return (float)(splitmix64(step_key + (unsigned long long)token_id) >> 40) * (1.0f / 16777216.0f);
 }
 
+// Range check of an index that a kernel has read from device memory (survivor lists, slots, move lists).  In the
+// ordinary build it costs nothing.  Built with -DOVGGT_BOUNDS_CHECK, an index outside [0, n) is not used: the access
+// is skipped and OVGGT_ERR_DEVICE_STATUS goes to the status word, which the next ovggt_cache_stats reports - no trap,
+// the kernel runs to its end.
+#ifdef OVGGT_BOUNDS_CHECK
+__device__ __forceinline__ bool index_ok(long long i, long long n, int* status) {
+  if (i >= 0 && i < n) return true;
+  if (status != nullptr) atomicCAS(status, 0, OVGGT_ERR_DEVICE_STATUS);
+  return false;
+}
+#else
+__device__ __forceinline__ bool index_ok(long long, long long, int*) { return true; }
+#endif
+
 // ---- block-wide primitives for a block of up to 1024 threads; `sh` holds >= 33 words.
 
 __device__ inline int block_sum_int(int x, int* sh) {

@@ -25,13 +25,15 @@ __device__ __forceinline__ void warp_copy_row(const uint4* __restrict__ src, uin
 // dst[j, :] = src[survivors[j], :] for K and V.  Work item 2j is K row j, 2j+1 is V row j.
 __global__ void __launch_bounds__(256) k_compact(const uint4* __restrict__ k_src, const uint4* __restrict__ v_src,
                                                  const int* __restrict__ survivors, int n_keep, int nvec,
-                                                 uint4* __restrict__ k_dst, uint4* __restrict__ v_dst) {
+                                                 uint4* __restrict__ k_dst, uint4* __restrict__ v_dst, int n_src,
+                                                 int* status) {
   const int lane = threadIdx.x & 31;
   const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
   for (int item = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5); item < 2 * n_keep;
        item += warps_total) {
     const int j = item >> 1;
     const int src = survivors[j];
+    if (!index_ok(src, n_src, status)) continue;
     if (item & 1) warp_copy_row(v_src + (size_t)src * nvec, v_dst + (size_t)j * nvec, nvec, lane);
     else          warp_copy_row(k_src + (size_t)src * nvec, k_dst + (size_t)j * nvec, nvec, lane);
   }
@@ -50,7 +52,7 @@ template <int DT>
 __global__ void __launch_bounds__(256) k_compact_colsum(const uint4* __restrict__ k_src, const uint4* __restrict__ v_src,
                                                         const int* __restrict__ survivors, int n_keep, int nvec,
                                                         uint4* __restrict__ k_dst, uint4* __restrict__ v_dst,
-                                                        float* __restrict__ part) {
+                                                        float* __restrict__ part, int n_src, int* status) {
   constexpr int VEC = VecOf<DT>::n;
   __shared__ __align__(16) float red[4][kCompactSumMaxVec * VEC];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -63,7 +65,9 @@ __global__ void __launch_bounds__(256) k_compact_colsum(const uint4* __restrict_
   for (int j0 = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5); j0 < n_keep; j0 += 2 * warps_total) {
     const int j1 = j0 + warps_total;
     const bool two = j1 < n_keep;
-    const int s0 = survivors[j0], s1 = two ? survivors[j1] : s0;
+    int s0 = survivors[j0], s1 = two ? survivors[j1] : s0;
+    if (!index_ok(s0, n_src, status)) s0 = 0;     // (checked build: a bad index is reported and row 0 copied instead)
+    if (!index_ok(s1, n_src, status)) s1 = 0;
     const uint4 *ka = k_src + (size_t)s0 * nvec, *va = v_src + (size_t)s0 * nvec;
     const uint4 *kb = k_src + (size_t)s1 * nvec, *vb = v_src + (size_t)s1 * nvec;
     uint4 uk[2][4], uv[2][4];
@@ -215,6 +219,8 @@ struct FillArgs {
   int max_moves;
   int* slot_meta;
   float* delta;                 // [kFillSlices, C] or nullptr
+  int rows_cap, n_meta;         // slots of the K/V buffer, entries of slot_meta (range checks of the checked build)
+  int* status;
 };
 
 template <int DT>
@@ -242,6 +248,9 @@ __device__ __forceinline__ void fill_holes_body(const FillArgs& A, int nvec) {
     for (int e = 0; e < VEC; ++e) acc[i][e] = 0.0f;
   for (int m = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5); m < n_moves; m += warps_total) {
     const int src = move_src[m], dst = move_dst[m];
+    if (!index_ok(src, A.rows_cap, A.status) || !index_ok(dst, A.rows_cap, A.status) ||
+        !index_ok(move_j[m], A.n_meta, A.status))
+      continue;
     for (int v0 = lane; v0 < nvec; v0 += 128) {
       uint4 uk[4], uv[4], uo[4];
 #pragma unroll
@@ -311,20 +320,156 @@ __global__ void __launch_bounds__(kFillThreads) k_fill_holes(uint4* __restrict__
                                                              const int* __restrict__ move_j,
                                                              const int* __restrict__ n_moves_ptr, int max_moves,
                                                              int nvec, int* __restrict__ slot_meta,
-                                                             float* __restrict__ delta /* [kFillSlices, C] or null */) {
-  const FillArgs A{k_cache, v_cache, move_src, move_dst, move_j, n_moves_ptr, max_moves, slot_meta, delta};
+                                                             float* __restrict__ delta /* [kFillSlices, C] or null */,
+                                                             int rows_cap, int n_meta, int* status) {
+  const FillArgs A{k_cache, v_cache, move_src, move_dst, move_j, n_moves_ptr, max_moves, slot_meta, delta,
+                   rows_cap, n_meta, status};
   fill_holes_body<DT>(A, nvec);
 }
 
-// The moves of several layers in one launch: blockIdx.y = position in the batch.  (A layer of the batch without
-// corrections to compute returns before the cluster barriers; all CTAs of its clusters do, so nobody is left waiting.)
-constexpr int kMaxFillBatch = 32;
-struct FillBatch {
-  FillArgs a[kMaxFillBatch];
+// Eq. 2 together with the move the previous step left behind.  The hole-filling move of step t and the append of
+// step t + 1 touch the same slots - the rows admitted at step t sit in slots >= B, exactly where frame t + 1 goes -
+// and nothing reads the cache in between, so one kernel does both and a step has one small launch less on its critical
+// path.  A warp owns new row j (slot n + j): if that slot still holds an admitted row (tail_move says which move), the
+// warp first carries it down to its destination, then writes the new K/V row over it; program order inside the warp
+// is all the ordering this needs.  Meta of the new rows and the corrections of the key column sums as in k_append and
+// k_fill_holes.  Launched as kFillSlices clusters of kFillClusterCtas CTAs.
+struct AppendFillArgs {
+  const uint4* k_new; const uint4* v_new;     // the frame's rows [M, C]
+  int M, n; long long frame_id;
+  uint4* k_cache; uint4* v_cache;
+  long long* ids; uint8_t* flags; float* stored; int* slot;   // meta of the layer, logical order
+  float* kmax2;                               // running bound of the key norms, or nullptr
+  int B;                                      // slots >= B may hold rows that still have to move
+  const int* tail_move; const int* move_dst; const int* move_j; const int* n_moves_ptr;   // nullptr: nothing pending
+  float* delta;                               // [kFillSlices, C] or nullptr
+  int* status;                                // where the checked build reports a bad move index
 };
+
+constexpr int kAppendFillThreads = 384;      // 16 clusters x 8 CTAs x 12 warps: a warp per row up to 1536 new rows
+
 template <int DT>
-__global__ void __launch_bounds__(kFillThreads) k_fill_holes_batched(const __grid_constant__ FillBatch batch, int nvec) {
-  fill_holes_body<DT>(batch.a[blockIdx.y], nvec);
+__global__ void __launch_bounds__(kAppendFillThreads) k_append_fill(const __grid_constant__ AppendFillArgs A, int nvec) {
+  constexpr int VEC = VecOf<DT>::n;
+  __shared__ __align__(16) float red[4][kCompactSumMaxVec * VEC];
+  __shared__ __align__(16) float cta_part[kCompactSumMaxVec * VEC];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int gtid = blockIdx.x * blockDim.x + threadIdx.x;
+  const int warps_total = (int)((gridDim.x * (unsigned)blockDim.x) >> 5);
+  const bool pending = A.tail_move != nullptr;
+  const bool sum = A.delta != nullptr;
+  float acc[4][VEC];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[i][e] = 0.0f;
+  for (int j = gtid >> 5; j < A.M; j += warps_total) {
+    const int s = A.n + j;                                   // the new row's slot
+    const bool tail = pending && s >= A.B && s - A.B < A.M;
+    // everything that does not depend on another load goes out first: the move's index, the number of moves, the
+    // new rows, and (speculatively, when a move may be pending for this slot) the rows that sit in the slot
+    int m = tail ? A.tail_move[s - A.B] : -1;
+    const int n_moves = tail ? min(*A.n_moves_ptr, A.M) : 0;
+    uint4 nk[4], nv[4], uk[4], uv[4], uo[4];
+    const int first = lane;                                  // rows longer than 128 vectors take further rounds below
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (first + 32 * i < nvec) {
+        nk[i] = ld_nc(A.k_new + (size_t)j * nvec + first + 32 * i);
+        nv[i] = ld_nc(A.v_new + (size_t)j * nvec + first + 32 * i);
+        if (tail) {   // (plain loads: these cache lines are rewritten by this very kernel)
+          uk[i] = A.k_cache[(size_t)s * nvec + first + 32 * i];
+          uv[i] = A.v_cache[(size_t)s * nvec + first + 32 * i];
+        }
+      }
+    // (a warp collective: every lane of the warp is here, whatever part of the row it holds; rows of up to 128
+    //  vectors only, which is all the bound is kept for)
+    if (A.kmax2 != nullptr) warp_key_norm_max(nk, nvec, lane, A.kmax2);
+    if (m >= n_moves) m = -1;
+    int dst = m >= 0 ? A.move_dst[m] : 0;
+    if (m >= 0 && (!index_ok(dst, A.B, A.status) || !index_ok(A.move_j[m], A.B, A.status))) m = -1;
+    for (int v0 = lane; v0 < nvec; v0 += 128) {
+      if (v0 != lane) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (v0 + 32 * i < nvec) {
+            nk[i] = ld_nc(A.k_new + (size_t)j * nvec + v0 + 32 * i);
+            nv[i] = ld_nc(A.v_new + (size_t)j * nvec + v0 + 32 * i);
+            if (m >= 0) {
+              uk[i] = A.k_cache[(size_t)s * nvec + v0 + 32 * i];
+              uv[i] = A.v_cache[(size_t)s * nvec + v0 + 32 * i];
+            }
+          }
+      }
+      if (m >= 0 && sum) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (v0 + 32 * i < nvec) uo[i] = A.k_cache[(size_t)dst * nvec + v0 + 32 * i];
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (v0 + 32 * i < nvec) {
+          if (m >= 0) {
+            A.k_cache[(size_t)dst * nvec + v0 + 32 * i] = uk[i];
+            A.v_cache[(size_t)dst * nvec + v0 + 32 * i] = uv[i];
+            if (sum) {
+              float a[VEC], b[VEC];
+              unpack<DT>(uk[i], a);
+              unpack<DT>(uo[i], b);
+#pragma unroll
+              for (int e = 0; e < VEC; ++e) acc[i][e] += a[e] - b[e];
+            }
+          }
+          A.k_cache[(size_t)s * nvec + v0 + 32 * i] = nk[i];
+          A.v_cache[(size_t)s * nvec + v0 + 32 * i] = nv[i];
+        }
+    }
+    if (lane == 0) {
+      if (m >= 0) A.slot[A.move_j[m]] = dst;
+      A.ids[s] = A.frame_id * (long long)A.M + j;
+      A.flags[s] = OVGGT_FLAG_EVICTABLE;
+      A.stored[s] = 0.0f;
+      A.slot[s] = s;
+    }
+  }
+  if (!sum) return;
+  // CTA fold in a fixed order: warps 8..11 park their sums in the four slots, 4..7 add theirs, 0..3 add theirs, then
+  // the four slots are added in order
+  auto park = [&](int slot_, bool add) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (lane + 32 * i < nvec)
+#pragma unroll
+        for (int e = 0; e < VEC; e += 4) {
+          float4* p = reinterpret_cast<float4*>(&red[slot_][(lane + 32 * i) * VEC + e]);
+          float4 t = make_float4(acc[i][e], acc[i][e + 1], acc[i][e + 2], acc[i][e + 3]);
+          if (add) {
+            const float4 o = *p;
+            t.x += o.x; t.y += o.y; t.z += o.z; t.w += o.w;
+          }
+          *p = t;
+        }
+  };
+  static_assert(kAppendFillThreads == 384, "the fold below is written for twelve warps");
+  if (warp >= 8) park(warp - 8, false);
+  __syncthreads();
+  if (warp >= 4 && warp < 8) park(warp - 4, true);
+  __syncthreads();
+  if (warp < 4) park(warp, true);
+  __syncthreads();
+  const int C = nvec * VEC;
+  for (int c = threadIdx.x; c < C; c += blockDim.x) cta_part[c] = ((red[0][c] + red[1][c]) + red[2][c]) + red[3][c];
+  cooperative_groups::cluster_group cluster = cooperative_groups::this_cluster();
+  cluster.sync();
+  const int ncta = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+  const int cid = (int)blockIdx.x / ncta;
+  for (int c = rank * 32 + (threadIdx.x & 31) + (threadIdx.x >> 5) * 32 * ncta; c < C;
+       c += 32 * ncta * (blockDim.x >> 5)) {
+    float t = 0.0f;
+    for (int q = 0; q < ncta; ++q) t += cluster.map_shared_rank(cta_part, q)[c];
+    A.delta[(size_t)cid * C + c] = t;
+  }
+  cluster.sync();   // no CTA may exit while others still read its shared memory
 }
 
 }  // namespace ovggt

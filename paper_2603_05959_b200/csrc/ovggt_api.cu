@@ -12,6 +12,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/ovggt.h"
 #include "attn_simt.cuh"
 #include "attn_tcgen05.cuh"
@@ -138,28 +140,29 @@ int launch_diversity_from_parts(const void* K, int rows, int C, int dtype, const
 
 // Compaction that also leaves per-CTA column sums of the keys it writes; *nparts = number of partial rows written.
 int launch_compact_colsum(const void* ks, const void* vs, const int* surv, int n_keep, int C, int dtype, void* kd,
-                          void* vd, float* part, int* nparts, cudaStream_t st) {
+                          void* vd, float* part, int* nparts, cudaStream_t st, int n_src, int* status) {
   *nparts = 0;
   if (n_keep <= 0) return OVGGT_OK;
   const int nvec = C * elem_bytes(dtype) / 16;
   const int grid = std::min((n_keep + 31) / 32, 148 * 8);   // four survivors (K and V rows) per warp
   if (dtype == kBF16)
     k_compact_colsum<kBF16><<<grid, 256, 0, st>>>((const uint4*)ks, (const uint4*)vs, surv, n_keep, nvec, (uint4*)kd,
-                                                  (uint4*)vd, part);
+                                                  (uint4*)vd, part, n_src, status);
   else
     k_compact_colsum<kF32><<<grid, 256, 0, st>>>((const uint4*)ks, (const uint4*)vs, surv, n_keep, nvec, (uint4*)kd,
-                                                 (uint4*)vd, part);
+                                                 (uint4*)vd, part, n_src, status);
   LAUNCHED();
   *nparts = grid;
   return OVGGT_OK;
 }
 
 int launch_compact(const void* ks, const void* vs, const int* surv, int n_keep, int C, int dtype, void* kd,
-                   void* vd, cudaStream_t st) {
+                   void* vd, cudaStream_t st, int n_src, int* status) {
   if (n_keep <= 0) return OVGGT_OK;
   const int nvec = C * elem_bytes(dtype) / 16;
   const int grid = std::min((2 * n_keep + 7) / 8, 148 * 8);
-  k_compact<<<grid, 256, 0, st>>>((const uint4*)ks, (const uint4*)vs, surv, n_keep, nvec, (uint4*)kd, (uint4*)vd);
+  k_compact<<<grid, 256, 0, st>>>((const uint4*)ks, (const uint4*)vs, surv, n_keep, nvec, (uint4*)kd, (uint4*)vd, n_src,
+                                  status);
   LAUNCHED();
   return OVGGT_OK;
 }
@@ -199,7 +202,8 @@ int launch_colsum(const void* K, int rows, int C, int dtype, float* part, float*
 
 // The hole-filling move (and, with delta, what it does to the key column sums).
 int launch_fill_holes(void* kc, void* vc, const int* msrc, const int* mdst, const int* mj, const int* n_moves, int max_moves,
-                      int C, int dtype, int* slot_meta, float* delta, cudaStream_t st) {
+                      int C, int dtype, int* slot_meta, float* delta, cudaStream_t st, int rows_cap, int n_meta,
+                      int* status) {
   const int nvec = C * elem_bytes(dtype) / 16;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(kFillSlices * kFillClusterCtas);
@@ -216,10 +220,10 @@ int launch_fill_holes(void* kc, void* vc, const int* msrc, const int* mdst, cons
   cudaError_t e;
   if (dtype == kBF16)
     e = cudaLaunchKernelEx(&cfg, k_fill_holes<kBF16>, (uint4*)kc, (uint4*)vc, msrc, mdst, mj, n_moves, max_moves, nvec,
-                           slot_meta, delta);
+                           slot_meta, delta, rows_cap, n_meta, status);
   else
     e = cudaLaunchKernelEx(&cfg, k_fill_holes<kF32>, (uint4*)kc, (uint4*)vc, msrc, mdst, mj, n_moves, max_moves, nvec,
-                           slot_meta, delta);
+                           slot_meta, delta, rows_cap, n_meta, status);
   if (e != cudaSuccess) return cuda_fail(e);
   LAUNCHED();
   return OVGGT_OK;
@@ -270,7 +274,9 @@ struct LayerState {
   float* colsum_part = nullptr;   // stable layout: [148 * 8, C] per-CTA column sums of the keys the last compaction wrote
   int colsum_nparts = 0;          // 0: not available (the next step sums the keys itself)
   // hole-filling layout
-  int *move_src = nullptr, *move_dst = nullptr, *move_j = nullptr, *n_moves_dev = nullptr;
+  int *move_src = nullptr, *move_dst = nullptr, *move_j = nullptr, *tail_move = nullptr, *n_moves_dev = nullptr;
+  bool moves_pending = false;     // the last compress left moves that the next append (or a flush) carries out
+  float* moves_delta = nullptr;   // where that move leaves its corrections of the key column sums, or nullptr
   float* ksum[2] = {nullptr, nullptr};   // [1 + kFillSlices, C]: the key column sums a step uses, then the move's corrections
   int kcur = 0;                   // which of the two the next diversity launch reads
   bool ksum_valid = false;        // ksum[kcur] describes the cached keys (else: recompute)
@@ -328,12 +334,16 @@ struct ProfScope {
   cudaStream_t st;
   bool on;
   ProfScope(ovggt_cache* h_, int cls, cudaStream_t st_) : h(h_), st(st_), on(h_->prof) {
+    static const char* const kNames[OVGGT_PROF_CLASSES] = {"ovggt append", "ovggt attention", "ovggt row norms",
+                                                           "ovggt diversity", "ovggt select", "ovggt compact"};
+    nvtxRangePushA(kNames[cls]);          // a named range around the launches of each class, for timeline tools
     if (!on) return;
     rec.cls = cls;
     if (cudaEventCreate(&rec.a) != cudaSuccess || cudaEventCreate(&rec.b) != cudaSuccess) { on = false; return; }
     cudaEventRecord(rec.a, st);
   }
   ~ProfScope() {
+    nvtxRangePop();
     if (!on) return;
     cudaEventRecord(rec.b, st);
     h->prof_recs.push_back(rec);
@@ -419,7 +429,7 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
     off[i++] = L.take((size_t)c->n_heads * 4);   // bound of the key norms
     if (fill) {
       for (int b = 0; b < 2; ++b) off[i++] = L.take(R * 4);                                  // slots
-      for (int b = 0; b < 3; ++b) off[i++] = L.take((size_t)M * 4);                          // move lists
+      for (int b = 0; b < 4; ++b) off[i++] = L.take((size_t)M * 4);                          // move lists
       for (int b = 0; b < 2; ++b) off[i++] = L.take((size_t)(1 + kFillSlices) * C * 4);      // column sums + corrections
     } else {
       off[i++] = L.take((size_t)148 * 8 * C * 4);   // column-sum partials of the compaction
@@ -445,6 +455,7 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
         S.move_src = reinterpret_cast<int*>(base + off[i++]);
         S.move_dst = reinterpret_cast<int*>(base + off[i++]);
         S.move_j = reinterpret_cast<int*>(base + off[i++]);
+        S.tail_move = reinterpret_cast<int*>(base + off[i++]);
         for (int b = 0; b < 2; ++b) S.ksum[b] = reinterpret_cast<float*>(base + off[i++]);
       } else {
         S.colsum_part = reinterpret_cast<float*>(base + off[i++]);
@@ -612,19 +623,65 @@ float* key_norm_bound(const ovggt_cache* h, const LayerState& S) {
   return (h->cfg.dtype == kBF16 && h->C * h->elem / 16 <= 128 && h->use_key_bound) ? S.kmax2 : nullptr;
 }
 
-// Eq. 2: the append itself.
+// Carry out the moves the layer's last compress left, now, with the stand-alone kernel (for whoever reads the K/V
+// buffer or the slots before the next append: export).
+int flush_moves(ovggt_cache* h, LayerState& S, cudaStream_t st) {
+  if (!S.moves_pending) return OVGGT_OK;
+  ProfScope ps(h, OVGGT_PROF_COMPACT, st);
+  int rc = launch_fill_holes(S.kbuf[S.kv], S.vbuf[S.kv], S.move_src, S.move_dst, S.move_j, S.n_moves_dev, h->M, h->C,
+                             h->cfg.dtype, S.slot[S.cur], S.moves_delta, st, S.budget + h->M, S.budget, h->status);
+  if (rc) return rc;
+  S.moves_pending = false;
+  S.moves_delta = nullptr;
+  return OVGGT_OK;
+}
+
+// Eq. 2: the append itself; in the hole-filling layout the same launch first carries out the moves the previous
+// compress left (they empty exactly the slots the new frame goes into).
 int enqueue_append(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st) {
   int rc = validate_attend(h, layer, io);
   if (rc) return rc;
   LayerState& S = h->layers[layer];
   h->last_stream = st;
   const int M = h->M, C = h->C, nvec = C * h->elem / 16, b = S.cur, kb = S.kv;
-  const int grid = std::min((2 * M + 7) / 8, 148 * 8);
   ProfScope ps(h, OVGGT_PROF_APPEND, st);
-  k_append<<<grid, 256, 0, st>>>((const uint4*)io->k, (const uint4*)io->v, M, nvec, S.n, (long long)io->frame_id,
-                                 (uint4*)S.kbuf[kb], (uint4*)S.vbuf[kb], S.ids[b], S.flags[b], S.stored[b], S.slot[b],
-                                 key_norm_bound(h, S));
+  if (!fill_layout(h)) {
+    const int grid = std::min((2 * M + 7) / 8, 148 * 8);
+    k_append<<<grid, 256, 0, st>>>((const uint4*)io->k, (const uint4*)io->v, M, nvec, S.n, (long long)io->frame_id,
+                                   (uint4*)S.kbuf[kb], (uint4*)S.vbuf[kb], S.ids[b], S.flags[b], S.stored[b], S.slot[b],
+                                   key_norm_bound(h, S));
+    LAUNCHED();
+    return OVGGT_OK;
+  }
+  AppendFillArgs A;
+  A.k_new = (const uint4*)io->k; A.v_new = (const uint4*)io->v;
+  A.M = M; A.n = S.n; A.frame_id = (long long)io->frame_id;
+  A.k_cache = (uint4*)S.kbuf[kb]; A.v_cache = (uint4*)S.vbuf[kb];
+  A.ids = S.ids[b]; A.flags = S.flags[b]; A.stored = S.stored[b]; A.slot = S.slot[b];
+  A.kmax2 = key_norm_bound(h, S);
+  A.B = S.budget;
+  const bool pending = S.moves_pending;
+  A.tail_move = pending ? S.tail_move : nullptr;
+  A.move_dst = S.move_dst; A.move_j = S.move_j; A.n_moves_ptr = S.n_moves_dev;
+  A.delta = pending ? S.moves_delta : nullptr;
+  A.status = h->status;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kFillSlices * kFillClusterCtas);
+  cfg.blockDim = dim3(kAppendFillThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = kFillClusterCtas;
+  attr.val.clusterDim.y = 1;
+  attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = h->cfg.dtype == kBF16 ? cudaLaunchKernelEx(&cfg, k_append_fill<kBF16>, A, nvec)
+                                        : cudaLaunchKernelEx(&cfg, k_append_fill<kF32>, A, nvec);
+  if (e != cudaSuccess) return cuda_fail(e);
   LAUNCHED();
+  S.moves_pending = false;
+  S.moves_delta = nullptr;
   return OVGGT_OK;
 }
 
@@ -772,7 +829,8 @@ CompressParams select_params(ovggt_cache* h, LayerState& S, const ovggt_frame_io
   P.status = h->status; P.n_keep_out = S.n_keep_dev;
   P.fill = fill_layout(h) ? 1 : 0;
   P.slot_src = S.slot[b]; P.slot_dst = S.slot[b ^ 1];
-  P.move_src = S.move_src; P.move_dst = S.move_dst; P.move_j = S.move_j; P.n_moves_out = S.n_moves_dev;
+  P.move_src = S.move_src; P.move_dst = S.move_dst; P.move_j = S.move_j; P.tail_move = S.tail_move;
+  P.n_moves_out = S.n_moves_dev;
   return P;
 }
 
@@ -800,12 +858,11 @@ bool move_leaves_corrections(const ovggt_cache* h, const LayerState& S) {
   return h->cfg.score_mode == OVGGT_SCORE_HYBRID && h->C * h->elem / 16 <= kCompactSumMaxVec && S.n == S.budget;
 }
 
-// The compress half.  Scores and selection go to st_sel.  What moves K/V rows goes to st_move: the stable gather
-// writes another buffer and may run beside an attention that still reads this one (st_move = st_sel); the
-// hole-filling move writes the buffer the attention reads, so it follows both (st_move = the attention's stream,
-// which first waits for st_sel).
-int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st_sel, cudaStream_t st_move,
+// The compress half on stream st.  The stable gather writes another buffer, so the whole half may run beside an
+// attention that still reads this one; the hole-filling moves are only recorded here (see enqueue_append).
+int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaStream_t st_sel,
                   const MirroredDecision* mirrored = nullptr) {
+  const cudaStream_t st_move = st_sel;
   int rc = validate_compress(h, layer, io, mirrored);
   if (rc) return rc;
   LayerState& S = h->layers[layer];
@@ -833,17 +890,13 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
   }
   const int n_keep = std::min(N, B);
   if (fill) {
+    // Some rows leave: the survivors above slot B have to move into the slots that open below it.  The selection
+    // kernel has left the pairs; the next append of this layer carries them out (flush_moves for other readers).
     S.ksum_valid = false;
-    if (N > B) {   // some rows leave: survivors above slot B move into the slots that open below it
-      if (st_move != st_sel) {
-        CK(cudaEventRecord(h->ev_join, st_sel));
-        CK(cudaStreamWaitEvent(st_move, h->ev_join, 0));
-      }
+    if (N > B) {
       const bool delta = move_leaves_corrections(h, S);
-      ProfScope ps(h, OVGGT_PROF_COMPACT, st_move);
-      rc = launch_fill_holes(S.kbuf[kb], S.vbuf[kb], S.move_src, S.move_dst, S.move_j, S.n_moves_dev, M, C, c.dtype,
-                             S.slot[b ^ 1], delta ? S.ksum[S.kcur ^ 1] + C : nullptr, st_move);
-      if (rc) return rc;
+      S.moves_pending = true;
+      S.moves_delta = delta ? S.ksum[S.kcur ^ 1] + C : nullptr;
       if (delta) {
         S.kcur ^= 1;
         S.ksum_valid = true;
@@ -855,9 +908,10 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
     S.colsum_nparts = 0;
     if (fuse)
       rc = launch_compact_colsum(S.kbuf[kb], S.vbuf[kb], S.surv, n_keep, C, c.dtype, S.kbuf[kb ^ 1], S.vbuf[kb ^ 1],
-                                 S.colsum_part, &S.colsum_nparts, st_move);
+                                 S.colsum_part, &S.colsum_nparts, st_move, N, h->status);
     else
-      rc = launch_compact(S.kbuf[kb], S.vbuf[kb], S.surv, n_keep, C, c.dtype, S.kbuf[kb ^ 1], S.vbuf[kb ^ 1], st_move);
+      rc = launch_compact(S.kbuf[kb], S.vbuf[kb], S.surv, n_keep, C, c.dtype, S.kbuf[kb ^ 1], S.vbuf[kb ^ 1], st_move, N,
+                          h->status);
     if (rc) return rc;
     S.kv = kb ^ 1;
   }
@@ -865,7 +919,7 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
   return OVGGT_OK;
 }
 
-// The compress half of every layer of the handle for one frame, in three launches instead of three per layer
+// The compress half of every layer of the handle for one frame, in two launches instead of two per layer
 // (hole-filling layout; the batched kernels take one parameter block per layer as kernel arguments).
 int compress_all_layers(ovggt_cache* h, const ovggt_frame_io* ios, cudaStream_t st) {
   const ovggt_config& c = h->cfg;
@@ -877,7 +931,7 @@ int compress_all_layers(ovggt_cache* h, const ovggt_frame_io* ios, cudaStream_t 
   }
   if (!fill_layout(h)) {                     // the stable gather has no batched kernels: layer by layer
     for (int l = 0; l < L; ++l) {
-      int rc = compress_impl(h, l, &ios[l], st, st);
+      int rc = compress_impl(h, l, &ios[l], st);
       if (rc) return rc;
     }
     return OVGGT_OK;
@@ -935,39 +989,17 @@ int compress_all_layers(ovggt_cache* h, const ovggt_frame_io* ios, cudaStream_t 
       CK(launch_cluster(k_compress_select_batched, dim3(ncta, cnt), ncta, smem, st, cb));
       LAUNCHED();
     }
-    // ---- the moves of the layers that evict
-    {
-      ProfScope ps(h, OVGGT_PROF_COMPACT, st);
-      FillBatch fb;
-      int nf = 0;
-      for (int i = 0; i < cnt; ++i) {
-        LayerState& S = h->layers[l0 + i];
-        S.ksum_valid = false;
-        if (S.n + M <= S.budget) continue;
-        const bool delta = move_leaves_corrections(h, S);
-        fb.a[nf++] = FillArgs{(uint4*)S.kbuf[S.kv], (uint4*)S.vbuf[S.kv], S.move_src, S.move_dst, S.move_j, S.n_moves_dev,
-                              M, S.slot[S.cur ^ 1], delta ? S.ksum[S.kcur ^ 1] + C : nullptr};
-        if (delta) {
-          S.kcur ^= 1;
-          S.ksum_valid = true;
-        }
-      }
-      if (nf > 0) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(kFillSlices * kFillClusterCtas, nf);
-        cfg.blockDim = dim3(kFillThreads);
-        cfg.stream = st;
-        cudaLaunchAttribute attr;
-        attr.id = cudaLaunchAttributeClusterDimension;
-        attr.val.clusterDim.x = kFillClusterCtas;
-        attr.val.clusterDim.y = 1;
-        attr.val.clusterDim.z = 1;
-        cfg.attrs = &attr;
-        cfg.numAttrs = 1;
-        cudaError_t e = c.dtype == kBF16 ? cudaLaunchKernelEx(&cfg, k_fill_holes_batched<kBF16>, fb, nvec)
-                                         : cudaLaunchKernelEx(&cfg, k_fill_holes_batched<kF32>, fb, nvec);
-        if (e != cudaSuccess) return cuda_fail(e);
-        LAUNCHED();
+    // ---- the moves of the layers that evict are left to each layer's next append
+    for (int i = 0; i < cnt; ++i) {
+      LayerState& S = h->layers[l0 + i];
+      S.ksum_valid = false;
+      if (S.n + M <= S.budget) continue;
+      const bool delta = move_leaves_corrections(h, S);
+      S.moves_pending = true;
+      S.moves_delta = delta ? S.ksum[S.kcur ^ 1] + C : nullptr;
+      if (delta) {
+        S.kcur ^= 1;
+        S.ksum_valid = true;
       }
     }
     for (int i = 0; i < cnt; ++i) close_compress(h, h->layers[l0 + i], &ios[l0 + i]);
@@ -985,7 +1017,7 @@ extern "C" int ovggt_layer_attend(ovggt_cache* h, int32_t layer, const ovggt_fra
 
 extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  return compress_impl(h, layer, io, st, st);
+  return compress_impl(h, layer, io, st);
 }
 
 extern "C" int ovggt_cache_anchor_decision(ovggt_cache* h, int64_t frame_id, int32_t* registered,
@@ -1002,7 +1034,7 @@ extern "C" int ovggt_camera_compress(ovggt_cache* h, int32_t layer, const ovggt_
   if (!h || !h->cfg.camera_head) return OVGGT_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const MirroredDecision d{registered != 0, demoted_frame};
-  return compress_impl(h, layer, io, st, st, &d);
+  return compress_impl(h, layer, io, st, &d);
 }
 
 extern "C" int ovggt_layers_compress(ovggt_cache* h, const ovggt_frame_io* ios, int32_t n_ios, void* stream) {
@@ -1024,25 +1056,23 @@ extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame
   }
   // Scoring and selection (Eq. 5-8) read the cache and the new rows but not the attention's output, so they run on
   // the handle's second, higher-priority stream beside the attention:
-  //   stream:  fork ........ append . fork' ........ attention ......................... join . [move]
-  //   side:         scores (diversity, norms) ....... [after fork'] selection [, gather] ..../
-  // The stable gather writes the other K/V buffer and stays on the side stream; the hole-filling move writes the
-  // buffer the attention reads and therefore follows the join on `stream`.
+  //   stream:  append (+ the previous step's moves) . fork ... attention ........................ join
+  //   side:                                            scores, selection [, stable gather] ....../
+  // The stable gather writes the other K/V buffer.  The hole-filling moves would write the buffer the attention
+  // reads; they wait for the next append of the layer, which has to touch the same slots anyway.
   rc = validate_attend(h, layer, io);
   if (rc) return rc;
   LayerState& S = h->layers[layer];
-  const bool fill = fill_layout(h);
+  rc = enqueue_append(h, layer, io, st);
+  if (rc) return rc;
   CK(cudaEventRecord(h->ev_fork, st));
   CK(cudaStreamWaitEvent(h->side, h->ev_fork, 0));
   rc = enqueue_scores(h, S, io, h->side);
-  if (rc == OVGGT_OK) S.scores_frame = io->frame_id;
-  if (rc == OVGGT_OK) rc = enqueue_append(h, layer, io, st);
   if (rc == OVGGT_OK) {
-    CK(cudaEventRecord(h->ev_app, st));
-    CK(cudaStreamWaitEvent(h->side, h->ev_app, 0));
+    S.scores_frame = io->frame_id;
     rc = enqueue_attention(h, layer, io, st);
   }
-  if (rc == OVGGT_OK) rc = compress_impl(h, layer, io, h->side, fill ? st : h->side);
+  if (rc == OVGGT_OK) rc = compress_impl(h, layer, io, h->side);
   // join: whatever happened, the caller's stream is ordered after the side work
   S.scores_frame = -1;
   h->last_stream = st;
@@ -1154,8 +1184,10 @@ extern "C" int ovggt_cache_export(ovggt_cache* h, int32_t layer, int64_t* token_
                                   void* k, void* v, int32_t* n_out) {
   int rc = check_layer(h, layer);
   if (rc) return rc;
-  const LayerState& S = h->layers[layer];
+  LayerState& S = h->layers[layer];
   if (S.pending) return OVGGT_ERR_FRAME_ORDER;
+  rc = flush_moves(h, S, h->last_stream);
+  if (rc) return rc;
   CK(cudaStreamSynchronize(h->last_stream));
   const int n = S.n, b = S.cur, kb = S.kv;
   const size_t row = (size_t)h->C * h->elem;
@@ -1242,6 +1274,8 @@ extern "C" int ovggt_cache_import(ovggt_cache* h, int32_t layer, const int64_t* 
   S.n = n;
   S.colsum_nparts = 0;          // the imported keys have not been summed
   S.ksum_valid = false;
+  S.moves_pending = false;      // (whatever was pending concerned rows that are gone)
+  S.moves_delta = nullptr;
   S.pending = false;
   S.n_prot_init = n_init;
   S.n_prot_hist = n_hist;
@@ -1270,6 +1304,8 @@ extern "C" int ovggt_cache_reset(ovggt_cache* h) {
     S.last_N = S.last_keep = 0;
     S.colsum_nparts = 0;
     S.ksum_valid = false;
+    S.moves_pending = false;
+    S.moves_delta = nullptr;
     S.since_refresh = 0;
     S.scores_frame = -1;
     CK(cudaMemset(S.kmax2, 0, (size_t)h->cfg.n_heads * 4));
@@ -1416,7 +1452,9 @@ extern "C" int ovggt_k_compact(const void* k_src, const void* v_src, const int32
   if (!k_src || !v_src || !survivors || !k_dst || !v_dst || n_keep < 0 || C < 1 || (C * elem_bytes(dtype)) % 16)
     return OVGGT_ERR_INVALID_ARG;
   if (!aligned16(k_src) || !aligned16(v_src) || !aligned16(k_dst) || !aligned16(v_dst)) return OVGGT_ERR_MISALIGNED;
-  return launch_compact(k_src, v_src, survivors, n_keep, C, dtype, k_dst, v_dst, static_cast<cudaStream_t>(stream));
+  // (the caller's source row count is not part of this call: the checked build has no bound to test against here)
+  return launch_compact(k_src, v_src, survivors, n_keep, C, dtype, k_dst, v_dst, static_cast<cudaStream_t>(stream),
+                        0x7FFFFFFF, nullptr);
 }
 
 extern "C" size_t ovggt_k_attention_scratch_bytes(int32_t M, int32_t N, int32_t n_heads) {

@@ -301,6 +301,7 @@ struct CompressParams {
   const int* slot_src;              // [n]
   int* slot_dst;                    // [<= B]
   int* move_src; int* move_dst; int* move_j;   // [<= M] each
+  int* tail_move;                   // [M]: for slot B + i, the index of the move that empties it, or -1
   int* n_moves_out;
 };
 
@@ -375,7 +376,10 @@ __device__ __forceinline__ void compress_select_body(const CompressParams& P, un
         id4[u] = P.ids_src[g];
         if (g < n) {
           st4[u] = P.stored_src[g];
-          if (P.fill) sl4[u] = P.slot_src[g];
+          if (P.fill) {
+            sl4[u] = P.slot_src[g];
+            if (!index_ok(sl4[u], P.B + P.M, P.status)) sl4[u] = g;
+          }
         }
       }
     }
@@ -534,13 +538,19 @@ __device__ __forceinline__ void compress_select_body(const CompressParams& P, un
         if (ssl[i] >= P.B && up_rank < M) {
           P.move_src[up_rank] = ssl[i];
           P.move_j[up_rank] = j;
+          if (ssl[i] - P.B < M) P.tail_move[ssl[i] - P.B] = up_rank;
           ++up_rank;
         }
         ++j;
-      } else if (ssl[i] < P.B && down_rank < M) {
-        P.move_dst[down_rank++] = ssl[i];
+      } else if (ssl[i] < P.B) {
+        if (down_rank < M) P.move_dst[down_rank++] = ssl[i];
+      } else if (ssl[i] - P.B < M) {
+        P.tail_move[ssl[i] - P.B] = -1;           // a row above slot B that leaves: its slot is simply free
       }
     }
+    // slots above B that no row occupies yet (the cache has just filled up) hold nothing to move
+    if (rank == 0)
+      for (int i = max(0, N - P.B) + tid; i < M; i += nthr) P.tail_move[i] = -1;
     if (rank == 0 && tid == 0) {
       // the two counts agree whenever the slots below min(N, B) were all occupied, which the layout guarantees
       const bool consistent = up_all == down_all && up_all <= M;

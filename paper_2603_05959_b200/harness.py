@@ -167,8 +167,15 @@ class Aggregator:
     confidence) come out of its heads after the last block.  `tap` and `after` as in ProjectionStack."""
 
     def __init__(self, cfg: gen.StreamConfig, device, compaction: int = B.COMPACT_FILL_HOLES,
-                 batched_compress: bool = True):
+                 batched_compress: bool = True, frame_attention: str = "library"):
+        """frame_attention: "library" runs the attention among the frame's own tokens on the library's tcgen05 kernel
+        (ovggt_k_attention with N = M: the same kernel that serves the cache); "torch" uses torch's SDPA."""
         self.batched_compress = batched_compress
+        self.frame_attention = frame_attention
+        M, H = cfg.tokens_per_frame, cfg.n_heads
+        self._fa_scratch = torch.empty(B.lib().ovggt_k_attention_scratch_bytes(M, M, H), dtype=torch.uint8, device=device)
+        self._fa_status = torch.zeros(16, dtype=torch.int32, device=device)
+        self._fa_out = torch.empty((M, cfg.dim), dtype=torch.bfloat16, device=device)
         assert cfg.dtype == gen.DTYPE_BF16
         self.cfg, self.device = cfg, device
         self.cache = B.OvggtCache.from_stream(cfg, device=device, compaction=compaction)
@@ -192,9 +199,15 @@ class Aggregator:
         resids, overrides = [], []
         for l in range(cfg.n_layers):
             w = self.blocks[l]["frame"]
-            qkv = (_layer_norm(x) @ w["qkv"]).view(M, 3, H, C // H).permute(1, 2, 0, 3)        # [3, H, M, d]
-            a = torch.nn.functional.scaled_dot_product_attention(qkv[0], qkv[1], qkv[2])       # within the frame
-            x = x + a.permute(1, 0, 2).reshape(M, C) @ w["o"]
+            qkv = _layer_norm(x) @ w["qkv"]
+            if self.frame_attention == "library":
+                fq, fk, fv = (qkv[:, i * C:(i + 1) * C].contiguous() for i in range(3))
+                a = B.k_attention(fq, fk, fv, H, out=self._fa_out, scratch=self._fa_scratch, status=self._fa_status,
+                                  stream=stream)
+            else:
+                q3 = qkv.view(M, 3, H, C // H).permute(1, 2, 0, 3)                               # [3, H, M, d]
+                a = torch.nn.functional.scaled_dot_product_attention(q3[0], q3[1], q3[2]).permute(1, 0, 2).reshape(M, C)
+            x = x + a @ w["o"]
             x = x + self._mlp(w, x)
             w = self.blocks[l]["global"]
             qkv = _layer_norm(x) @ w["qkv"]

@@ -110,6 +110,16 @@ def test_null_handle_and_strerror(lib):
     assert lib.ovggt_k_select(None, None, 0, 0, 1, None, None, None) == -1
 
 
+def test_checked_build_compiles_and_exports_the_same_symbols():
+    """The variant with range-checked indices (-DOVGGT_BOUNDS_CHECK) is the same library: it must build for sm_100a
+    and export every declared symbol."""
+    path = build_mod.build(checked=True)
+    assert path.endswith("libovggt_checked.so") and os.path.exists(path)
+    checked = C.CDLL(path)
+    for n in declared_symbols():
+        assert hasattr(checked, n), n
+
+
 def test_build_refuses_an_attention_kernel_with_another_launch_register_count():
     """setmaxnreg moves registers inside the pool the CTA is launched with; the build checks ptxas' launch count
     against the count the warpgroup budgets in the source were written for."""
