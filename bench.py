@@ -489,7 +489,8 @@ def run_stack(args) -> None:
     uuid = str(torch.cuda.get_device_properties(dev).uuid)
     sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
     sampler.start()
-    model = H.ProjectionStack(cfg, dev) if args.config == "c3" else H.Aggregator(cfg, dev)
+    model = H.ProjectionStack(cfg, dev, matmul=args.scaffold) if args.config == "c3" else \
+        H.Aggregator(cfg, dev, matmul=args.scaffold, frame_attention=args.scaffold)
     stream = torch.cuda.current_stream()
     fill = -(-Bud // M) + 1
     pool = min(args.pool, 24)
@@ -548,6 +549,15 @@ def run_stack(args) -> None:
     eb = cfg.elem_bytes
     alg_bytes = {"append": 8 * M * C * eb, "row_norms": M * C * eb + 4 * M,
                  "diversity": Bud * C * eb + 4 * Bud + M * C * eb + 4 * M, "select": 4 * N + N + 4 * Bud}
+    # c4 compresses all layers with one call at the end of the frame: its diversity and select launches are the batched
+    # ones (one launch group per frame covering L layers), so their algorithmic bytes are L layers' worth
+    n_frames_prof = min(K, 10)
+    for name in ("diversity", "select"):
+        if prof[name]["count"] == n_frames_prof:
+            alg_bytes[name] *= L
+    kernels = kernel_table(prof, alg_bytes, peaks, clocks.get("sm_mhz"))
+    for name in ("diversity", "select"):
+        kernels[name]["layers_per_launch_group"] = L if prof[name]["count"] == n_frames_prof else 1
     line = {"metric": METRIC, "value": K / (total_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": K, "warmup": W,
             "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
@@ -557,14 +567,15 @@ def run_stack(args) -> None:
                       "visited in turn; no explicit flush"}),
             "time_split_ms_per_frame": {"all": all_ms, "library": lib_ms, "scaffold": all_ms - lib_ms,
                                         "library_layer_steps_per_s": L / (lib_ms * 1e-3),
-                                        "note": "events around every library call in a separate pass of "
-                                                f"{n_split} frames; scaffold = torch matmuls / LayerNorm / frame "
-                                                "attention / MLP with random-init weights"},
+                                        "note": "events around every call of the streaming step's entry points in a "
+                                                f"separate pass of {n_split} frames; scaffold = projections, MLPs, "
+                                                "LayerNorm, frame attention with random-init weights "
+                                                f"(matmuls and frame attention on: {args.scaffold})"},
             "e2e": None, "gpu_launches": int(launches), "launches_per_step": launches / K, "clocks": clocks,
             "roofline": {"kernel": "k_attn_tcgen05", "bound": "tensor", "achieved": achieved, "peak": peak,
                          "unit": "TFLOP/s", "frac": achieved / peak, "peak_kind": f"{peak_kind} burst cuBLAS bf16 peak",
                          "traffic": None, "algorithmic_flops": attn_flops, "launch_ms": attn_ms},
-            "kernels": kernel_table(prof, alg_bytes, peaks, clocks.get("sm_mhz")),
+            "kernels": kernels,
             "ms_per_frame": H.flatness(per_frame)}
     if not args.no_cpu_baseline:
         # the oracle's share is one layer-step of this shape; a frame is L of them
@@ -687,6 +698,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference", "launch-check"])
     ap.add_argument("--config", default="c2", choices=sorted(WORKLOADS))
     ap.add_argument("--compaction", default="fill", choices=["fill", "stable"])
+    ap.add_argument("--scaffold", default="library", choices=["library", "torch"],
+                    help="c3 / c4: projections, MLPs and frame attention on the library's tcgen05 kernels or on torch")
     ap.add_argument("--streams", type=int, default=0, help="independent streams in rotation (0: enough to exceed L2)")
     ap.add_argument("--pool", type=int, default=160, help="distinct frames kept on the device (cycled beyond)")
     ap.add_argument("--e2e-steps", type=int, default=200)

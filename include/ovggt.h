@@ -327,6 +327,13 @@ int ovggt_k_key_norm_bound(const void* K, int32_t rows, int32_t n_heads, float* 
 int ovggt_k_attention_bounded(const void* q, const void* k, const void* v, int32_t M, int32_t N, int32_t n_heads,
                               void* out, void* scratch, int32_t* device_status, const float* kmax2, void* stream);
 
+/* Not a step of the paper's path: the dense products a model wraps around it (QKV and output projections, MLP), so
+ * that the multi-layer workloads can run their scaffold on a hand-written tcgen05 kernel as well.
+ * C [M, N] = A [M, K] x B [K, N], all bf16 row-major, fp32 accumulation, device pointers, 16-byte aligned; K must be a
+ * multiple of 64 and N of 8 (OVGGT_ERR_UNSUPPORTED otherwise).  device_status: device int, as for ovggt_k_attention. */
+int ovggt_k_gemm_bf16(const void* A, const void* B, int32_t M, int32_t N, int32_t K, void* C, int32_t* device_status,
+                      void* stream);
+
 #ifdef __cplusplus
 }
 #endif

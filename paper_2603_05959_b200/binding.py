@@ -31,7 +31,7 @@ EXPORTED = [
     "ovggt_cache_profile_enable", "ovggt_cache_profile_read", "ovggt_cache_set_overlap", "ovggt_cache_set_key_bound",
     "ovggt_strerror", "ovggt_last_cuda_error", "ovggt_k_row_norms", "ovggt_k_diversity_scratch_bytes",
     "ovggt_k_diversity", "ovggt_k_diversity_static", "ovggt_k_select", "ovggt_k_compact", "ovggt_k_attention_scratch_bytes",
-    "ovggt_k_attention", "ovggt_k_key_norm_bound", "ovggt_k_attention_bounded",
+    "ovggt_k_attention", "ovggt_k_key_norm_bound", "ovggt_k_attention_bounded", "ovggt_k_gemm_bf16",
 ]
 
 
@@ -120,6 +120,7 @@ def lib():
         L.ovggt_k_attention_scratch_bytes.argtypes = [i32, i32, i32]
         L.ovggt_k_attention.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp]
         L.ovggt_k_key_norm_bound.argtypes = [vp, i32, i32, vp, vp]
+        L.ovggt_k_gemm_bf16.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
         L.ovggt_k_attention_bounded.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp]
         _LIB = L
     return _LIB
@@ -392,6 +393,22 @@ def k_compact(k_src, v_src, survivors, k_dst=None, v_dst=None, stream=None):
     _check(lib().ovggt_k_compact(_dptr(k_src), _dptr(v_src), _dptr(survivors), n_keep, Cdim, dtype,
                                  _dptr(k_dst), _dptr(v_dst), _stream_ptr(stream)), "ovggt_k_compact")
     return k_dst, v_dst
+
+
+def k_gemm_bf16(a: torch.Tensor, b: torch.Tensor, out=None, status=None, stream=None) -> torch.Tensor:
+    """out [M, N] = a [M, K] @ b [K, N], bf16 in and out, on the library's tcgen05 GEMM."""
+    assert a.dtype == torch.bfloat16 and b.dtype == torch.bfloat16 and a.shape[1] == b.shape[0]
+    M, K = a.shape
+    N = b.shape[1]
+    out = torch.empty((M, N), dtype=torch.bfloat16, device=a.device) if out is None else out
+    own = status is None
+    if own:
+        status = torch.zeros(16, dtype=torch.int32, device=a.device)
+    _check(lib().ovggt_k_gemm_bf16(_dptr(a), _dptr(b), M, N, K, _dptr(out), _dptr(status), _stream_ptr(stream)),
+           "ovggt_k_gemm_bf16")
+    if own:
+        _check(int(status[0].item()), "ovggt_k_gemm_bf16 (device status)")
+    return out
 
 
 def k_key_norm_bound(k: torch.Tensor, n_heads: int, stream=None) -> torch.Tensor:

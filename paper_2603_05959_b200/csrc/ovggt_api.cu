@@ -19,6 +19,7 @@
 #include "attn_tcgen05.cuh"
 #include "common.cuh"
 #include "compact_kernels.cuh"
+#include "gemm_tcgen05.cuh"
 #include "score_kernels.cuh"
 #include "select_kernel.cuh"
 
@@ -566,6 +567,7 @@ extern "C" int ovggt_cache_create(const ovggt_config* cfg, ovggt_cache** out) {
   if (e == cudaSuccess) e = cudaMemset(h->ksum, 0, colsum_scratch_bytes(h->C));   // (its arrival counters)
   for (LayerState& S : h->layers)
     if (e == cudaSuccess) e = cudaMemset(S.kmax2, 0, (size_t)cfg->n_heads * 4);
+
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     delete h;
@@ -1489,6 +1491,17 @@ extern "C" int ovggt_k_attention_bounded(const void* q, const void* k, const voi
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return OVGGT_ERR_MISALIGNED;
   return launch_attention(q, k, v, M, N, n_heads, kBF16, out, scratch, device_status, static_cast<cudaStream_t>(stream),
                           nullptr, kmax2);
+}
+
+extern "C" int ovggt_k_gemm_bf16(const void* A, const void* Bm, int32_t M, int32_t N, int32_t K, void* C,
+                                 int32_t* device_status, void* stream) {
+  if (!A || !Bm || !C || !device_status || M < 1 || N < 1 || K < 1) return OVGGT_ERR_INVALID_ARG;
+  if (K % 64 != 0 || N % 8 != 0) return OVGGT_ERR_UNSUPPORTED;
+  if (!aligned16(A) || !aligned16(Bm) || !aligned16(C)) return OVGGT_ERR_MISALIGNED;
+  int rc = gemm_tcgen05_launch(A, Bm, C, M, N, K, device_status, static_cast<cudaStream_t>(stream));
+  if (rc == OVGGT_OK) g_launches.fetch_add(1);
+  if (rc == OVGGT_ERR_CUDA) g_last_cuda_error.store(attn_tcgen05_last_error());
+  return rc;
 }
 
 // ------------------------------------------------------------------ allocation-free diversity

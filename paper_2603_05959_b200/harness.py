@@ -108,6 +108,24 @@ class _Timer:
         return t
 
 
+class _Matmul:
+    """x @ W of the scaffold: torch's matmul, or the library's own tcgen05 GEMM (ovggt_k_gemm_bf16).  Either way it is
+    scaffold time, not the streaming step's."""
+
+    def __init__(self, kind: str, device):
+        assert kind in ("torch", "library")
+        self.kind = kind
+        self.status = torch.zeros(16, dtype=torch.int32, device=device)
+
+    def __call__(self, x: torch.Tensor, w: torch.Tensor, stream=None) -> torch.Tensor:
+        if self.kind == "torch":
+            return x @ w
+        return B.k_gemm_bf16(x.contiguous(), w, status=self.status, stream=stream)
+
+    def check(self) -> None:
+        assert int(self.status[0].item()) == 0
+
+
 def _randn(shape, std, device, dtype, gen_):
     return (torch.randn(shape, generator=gen_, device=device, dtype=torch.float32) * std).to(dtype)
 
@@ -119,9 +137,10 @@ class ProjectionStack:
     library input and may return priorities to rank instead of the library's own (teacher forcing in the tests);
     `after(t, l, out)` sees the attention output of every library call."""
 
-    def __init__(self, cfg: gen.StreamConfig, device, compaction: int = B.COMPACT_FILL_HOLES):
+    def __init__(self, cfg: gen.StreamConfig, device, compaction: int = B.COMPACT_FILL_HOLES, matmul: str = "library"):
         assert cfg.dtype == gen.DTYPE_BF16
         self.cfg, self.device = cfg, device
+        self.mm = _Matmul(matmul, device)
         self.cache = B.OvggtCache.from_stream(cfg, device=device, compaction=compaction)
         g = torch.Generator(device=device)
         g.manual_seed(cfg.seed)
@@ -138,7 +157,7 @@ class ProjectionStack:
         C = self.cfg.dim
         for l in range(self.cfg.n_layers):
             # embeddings are N(0, 1) over 1024 columns and the weights N(0, 0.02): q, k, v come out near N(0, 0.4)
-            qkv = x @ self.w_qkv[l]
+            qkv = self.mm(x, self.w_qkv[l], stream)
             q, k, v = (qkv[:, i * C:(i + 1) * C].contiguous() for i in range(3))
             ov = self.tap(t, l, q, k, v, resid[l]) if self.tap else None
             run = lambda: self.cache.layer_step(l, t, q, k, v, resid[l], conf, rho, score_override=ov, out=self.out,
@@ -146,10 +165,11 @@ class ProjectionStack:
             lib(run) if lib else run()
             if self.after:
                 self.after(t, l, self.out)
-            x = x + self.out @ self.w_o[l]
+            x = x + self.mm(self.out, self.w_o[l], stream)
         return x
 
     def destroy(self) -> None:
+        self.mm.check()
         self.cache.destroy()
 
 
@@ -167,10 +187,12 @@ class Aggregator:
     confidence) come out of its heads after the last block.  `tap` and `after` as in ProjectionStack."""
 
     def __init__(self, cfg: gen.StreamConfig, device, compaction: int = B.COMPACT_FILL_HOLES,
-                 batched_compress: bool = True, frame_attention: str = "library"):
+                 batched_compress: bool = True, frame_attention: str = "library", matmul: str = "library"):
         """frame_attention: "library" runs the attention among the frame's own tokens on the library's tcgen05 kernel
-        (ovggt_k_attention with N = M: the same kernel that serves the cache); "torch" uses torch's SDPA."""
+        (ovggt_k_attention with N = M: the same kernel that serves the cache); "torch" uses torch's SDPA.
+        matmul: "library" runs every projection and MLP product on ovggt_k_gemm_bf16; "torch" on torch's matmul."""
         self.batched_compress = batched_compress
+        self.mm = _Matmul(matmul, device)
         self.frame_attention = frame_attention
         M, H = cfg.tokens_per_frame, cfg.n_heads
         self._fa_scratch = torch.empty(B.lib().ovggt_k_attention_scratch_bytes(M, M, H), dtype=torch.uint8, device=device)
@@ -189,8 +211,8 @@ class Aggregator:
         self.tap: Optional[Callable] = None
         self.after: Optional[Callable] = None
 
-    def _mlp(self, w, h):
-        return torch.nn.functional.gelu(_layer_norm(h) @ w["fc1"]) @ w["fc2"]
+    def _mlp(self, w, h, stream=None):
+        return self.mm(torch.nn.functional.gelu(self.mm(_layer_norm(h), w["fc1"], stream)), w["fc2"], stream)
 
     def frame(self, t: int, x: torch.Tensor, conf: torch.Tensor, rho: float, stream,
               lib: Optional[_Timer] = None) -> torch.Tensor:
@@ -199,7 +221,7 @@ class Aggregator:
         resids, overrides = [], []
         for l in range(cfg.n_layers):
             w = self.blocks[l]["frame"]
-            qkv = _layer_norm(x) @ w["qkv"]
+            qkv = self.mm(_layer_norm(x), w["qkv"], stream)
             if self.frame_attention == "library":
                 fq, fk, fv = (qkv[:, i * C:(i + 1) * C].contiguous() for i in range(3))
                 a = B.k_attention(fq, fk, fv, H, out=self._fa_out, scratch=self._fa_scratch, status=self._fa_status,
@@ -207,17 +229,17 @@ class Aggregator:
             else:
                 q3 = qkv.view(M, 3, H, C // H).permute(1, 2, 0, 3)                               # [3, H, M, d]
                 a = torch.nn.functional.scaled_dot_product_attention(q3[0], q3[1], q3[2]).permute(1, 0, 2).reshape(M, C)
-            x = x + a @ w["o"]
-            x = x + self._mlp(w, x)
+            x = x + self.mm(a, w["o"], stream)
+            x = x + self._mlp(w, x, stream)
             w = self.blocks[l]["global"]
-            qkv = _layer_norm(x) @ w["qkv"]
+            qkv = self.mm(_layer_norm(x), w["qkv"], stream)
             q, k, v = (qkv[:, i * C:(i + 1) * C].contiguous() for i in range(3))
             att = lambda: self.cache.layer_attend(l, t, q, k, v, out=self.out, stream=stream)
             lib(att) if lib else att()
             if self.after:
                 self.after(t, l, self.out)
-            h = x + self.out @ w["o"]
-            r = self._mlp(w, h).contiguous()
+            h = x + self.mm(self.out, w["o"], stream)
+            r = self._mlp(w, h, stream).contiguous()
             ov = self.tap(t, l, q, k, v, r) if self.tap else None
             if self.batched_compress:
                 resids.append(r)
@@ -233,6 +255,7 @@ class Aggregator:
         return x
 
     def destroy(self) -> None:
+        self.mm.check()
         self.cache.destroy()
 
 

@@ -108,6 +108,7 @@ def test_null_handle_and_strerror(lib):
     assert lib.ovggt_kernel_launches() == 0
     assert lib.ovggt_k_row_norms(None, 1, 64, 0, None, None) == -1
     assert lib.ovggt_k_select(None, None, 0, 0, 1, None, None, None) == -1
+    assert lib.ovggt_k_gemm_bf16(None, None, 1, 8, 64, None, None, None) == -1
 
 
 def test_checked_build_compiles_and_exports_the_same_symbols():

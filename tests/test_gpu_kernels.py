@@ -216,6 +216,19 @@ def test_attention_bf16_peaked_logits_other_shapes(M, N, H, bounded):
     assert_attention_close_relative(got[rows], orc.attention(q, k, v, H, 64, rows=rows), f"{M}x{N}")
 
 
+@pytest.mark.parametrize("M,N,K", [(128, 128, 64), (5, 8, 64), (130, 136, 192), (1374, 3072, 1024), (1041, 1024, 4096)])
+def test_gemm_bf16_against_the_plain_product(M, N, K):
+    """The scaffold GEMM (not a step of the paper's path): C = A B against the definition in fp64 (numpy's matmul on
+    the same bf16-rounded inputs); bf16 output: half an ulp of the result plus fp32 accumulation error."""
+    a, b = rnd((M, K), gen.DTYPE_BF16, 3 + M), rnd((K, N), gen.DTYPE_BF16, 4 + N, scale=0.05)
+    got = B.k_gemm_bf16(dev(a, 1), dev(b, 1)).float().cpu().numpy()
+    ref = a.astype(np.float64) @ b.astype(np.float64)
+    np.testing.assert_allclose(got, ref, rtol=2 ** -8, atol=1e-3 * np.abs(ref).max())
+    with pytest.raises(B.OvggtError) as e:                    # K must be a multiple of 64
+        B.k_gemm_bf16(dev(a[:, :K - 8], 1), dev(b[:K - 8], 1))
+    assert e.value.code == -10
+
+
 def test_attention_is_deterministic():
     q, k, v = (dev(rnd(s, 1, i), 1) for i, s in enumerate(((500, 256), (3000, 256), (3000, 256))))
     a, b = B.k_attention(q, k, v, 4), B.k_attention(q, k, v, 4)
