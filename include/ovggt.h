@@ -68,8 +68,8 @@ enum { OVGGT_SCORE_HYBRID = 0, OVGGT_SCORE_RESIDUAL_STORED = 1, OVGGT_SCORE_RAND
 enum { OVGGT_FLAG_EVICTABLE = 0, OVGGT_FLAG_INIT = 1, OVGGT_FLAG_HIST = 2 };
 /* Where surviving K/V rows live after Eq. 8 (the paper fixes the survivor set, not a layout):
  *  FILL_HOLES     one K/V buffer per layer; the rows admitted from the new frame are copied into the slots the
- *                 evicted rows leave (at most M rows move per step); logical (token id) order is kept in per-row
- *                 meta and restored by ovggt_cache_export.  Attention reads the buffer front to back: the order of
+ *                 evicted rows leave (at most M rows move per step, inside the layer's next append); logical
+ *                 (token id) order is kept in per-row meta and restored by ovggt_cache_export.  Attention reads the buffer front to back: the order of
  *                 cached rows does not change its result beyond fp32 summation order.
  *  STABLE_GATHER  two K/V buffers per layer; every survivor is copied, in token order, into the other buffer
  *                 (B rows move per step; rows lie in token order on the device). */
@@ -153,9 +153,10 @@ int ovggt_layer_compress(ovggt_cache* cache, int32_t layer, const ovggt_frame_io
  * given at create): ios [n_ios], n_ios = n_layers, ios[l] describing layer l's pending frame (all with the same
  * frame_id; conf and rho are taken from ios[0]).  This is the call for a model whose anchor inputs exist only after
  * its heads have run: attend layer by layer, then compress all layers together.  In the hole-filling layout the
- * scores, the selection and the moves of up to 32 layers each go out as one launch (blockIdx.y = layer; one
- * thread-block cluster per layer for the selection), so the small per-layer kernels fill the GPU together; in the
- * stable-gather layout the layers are compressed one after the other.  All layers are checked before anything
+ * scores and the selection of up to 32 layers each go out as one launch (blockIdx.y = layer; one thread-block
+ * cluster per layer for the selection), so the small per-layer kernels fill the GPU together, and the moves of each
+ * layer ride in that layer's next append as always; in the stable-gather layout the layers are compressed one after
+ * the other.  All layers are checked before anything
  * changes; results are those of n_layers single calls. */
 int ovggt_layers_compress(ovggt_cache* cache, const ovggt_frame_io* ios, int32_t n_ios, void* stream);
 
@@ -177,8 +178,9 @@ int ovggt_camera_compress(ovggt_cache* camera, int32_t layer, const ovggt_frame_
  * read the cache and the new rows but not the attention's output, so they are enqueued on a second stream that the
  * handle owns (a host object, created by ovggt_cache_create), forked from and joined back into `stream` with
  * events, and run beside the attention; so does the stable gather, which writes another buffer.  The hole-filling
- * move writes the buffer the attention reads and follows the join on `stream`.  For the caller the call is still
- * asynchronous and ordered on `stream` alone. */
+ * moves would write the buffer the attention reads: the selection only records them, and the layer's next append
+ * (which touches the same slots) carries them out first; ovggt_cache_export flushes them.  For the caller the call
+ * is still asynchronous and ordered on `stream` alone. */
 int ovggt_layer_step(ovggt_cache* cache, int32_t layer, const ovggt_frame_io* io, void* stream);
 
 /* Turn the overlap of ovggt_layer_step off (0) or on (non-zero, the default): off, the two halves run one after the

@@ -316,7 +316,7 @@ struct ovggt_cache {
   // ovggt_layer_step scores the cache (diversity, residual norms) on a second, higher-priority stream while the
   // attention runs: the scores do not depend on the attention.  Host objects only; absent if creation failed.
   cudaStream_t side = nullptr;
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_app = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   bool overlap = true;            // ovggt_cache_set_overlap
   bool use_key_bound = true;      // ovggt_cache_set_key_bound
   // optional per-kernel-class timing (host-side CUDA events; no device memory)
@@ -537,13 +537,12 @@ extern "C" int ovggt_cache_create(const ovggt_config* cfg, ovggt_cache** out) {
     if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess ||
         cudaStreamCreateWithPriority(&h->side, cudaStreamNonBlocking, hi) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess ||
-        cudaEventCreateWithFlags(&h->ev_app, cudaEventDisableTiming) != cudaSuccess) {
+        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess) {
       if (h->ev_fork) cudaEventDestroy(h->ev_fork);
       if (h->ev_join) cudaEventDestroy(h->ev_join);
       if (h->side) cudaStreamDestroy(h->side);
       h->side = nullptr;
-      h->ev_fork = h->ev_join = h->ev_app = nullptr;
+      h->ev_fork = h->ev_join = nullptr;
       (void)cudaGetLastError();
     }
   }
@@ -596,7 +595,6 @@ extern "C" int ovggt_cache_destroy(ovggt_cache* h) {
     cudaStreamDestroy(h->side);
     cudaEventDestroy(h->ev_fork);
     cudaEventDestroy(h->ev_join);
-    cudaEventDestroy(h->ev_app);
   }
   delete h;
   return OVGGT_OK;
