@@ -25,6 +25,9 @@ class OrcConfig(C.Structure):
     ]
 
 
+SCORE_HYBRID, SCORE_RESIDUAL_STORED, SCORE_RANDOM, SCORE_QK = 0, 1, 2, 3
+
+
 def _f32(a):
     return np.ascontiguousarray(a, dtype=np.float32)
 
@@ -60,6 +63,8 @@ def lib():
         L.orc_export.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_uint8),
                                  C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_float)]
         L.orc_residual_norms.argtypes = [C.POINTER(C.c_float), C.c_int32, C.c_int32, C.POINTER(C.c_double)]
+        L.orc_qk_scores.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_int32, C.c_int32, C.c_int32,
+                                    C.POINTER(C.c_double)]
         L.orc_smooth.argtypes = [C.POINTER(C.c_double), C.c_int32, C.c_int32, C.c_int32, C.c_double,
                                  C.POINTER(C.c_double)]
         L.orc_diversity.argtypes = [C.POINTER(C.c_float), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
@@ -96,6 +101,16 @@ def residual_norms(R: np.ndarray) -> np.ndarray:
     R = _f32(R)
     s = np.empty(R.shape[0], dtype=np.float64)
     lib().orc_residual_norms(_ptr(R, C.c_float), R.shape[0], R.shape[1], _ptr(s, C.c_double))
+    return s
+
+
+def qk_scores(Q: np.ndarray, K: np.ndarray, n_heads: int) -> np.ndarray:
+    """Supp. D, query-key criterion: mean scaled logit each of the frame's keys gets from the frame's queries."""
+    Q, K = _f32(Q), _f32(K)
+    assert Q.shape == K.shape and Q.shape[1] % n_heads == 0
+    s = np.empty(Q.shape[0], dtype=np.float64)
+    lib().orc_qk_scores(_ptr(Q, C.c_float), _ptr(K, C.c_float), Q.shape[0], n_heads, Q.shape[1] // n_heads,
+                        _ptr(s, C.c_double))
     return s
 
 
@@ -240,8 +255,11 @@ class OracleLayer:
         return out
 
     def compress(self, resid, conf=None, rho=float("nan"), score_override=None):
-        resid = _f32(resid)
-        assert resid.shape == (self.M, self.C)
+        if resid is None:   # SCORE_QK reads the queries kept by attend() instead
+            assert self.cfg.score_mode == SCORE_QK
+        else:
+            resid = _f32(resid)
+            assert resid.shape == (self.M, self.C)
         conf_a = None if conf is None else _f32(conf)
         N = self.n_rows
         ov = None if score_override is None else _f32(score_override)

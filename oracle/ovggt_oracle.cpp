@@ -30,6 +30,24 @@ extern "C" void orc_residual_norms(const float* R, int32_t M, int32_t C, double*
   }
 }
 
+/* ------------------------------------------------------------------ Supp. D, query-key criterion */
+extern "C" void orc_qk_scores(const float* Q, const float* K, int32_t M, int32_t n_heads, int32_t head_dim,
+                              double* s) {
+  const int32_t C = n_heads * head_dim;
+  const double scale = 1.0 / std::sqrt((double)head_dim);
+  for (int32_t j = 0; j < M; ++j) {
+    double total = 0.0;
+    for (int32_t h = 0; h < n_heads; ++h)
+      for (int32_t i = 0; i < M; ++i) {
+        double logit = 0.0;
+        for (int32_t e = 0; e < head_dim; ++e)
+          logit += (double)Q[(size_t)i * C + h * head_dim + e] * (double)K[(size_t)j * C + h * head_dim + e];
+        total += logit * scale;
+      }
+    s[j] = total / ((double)M * (double)n_heads);
+  }
+}
+
 /* ------------------------------------------------------------------ Eq. 6
  * G is the 3x3 Gaussian with sigma = 1, G[dy][dx] proportional to
  * exp(-(dx^2 + dy^2) / 2), normalised to sum 1.  Outside the map the nearest
@@ -219,6 +237,7 @@ struct orc_state {
   std::vector<uint8_t> flags;
   std::vector<float> stored;   /* smoothed activation score each row had when it was new */
   std::vector<float> k, v;     /* [rows, C] */
+  std::vector<float> q_frame;  /* [M, C] queries of the pending frame (ORC_SCORE_QK only) */
   std::deque<int64_t> anchors; /* active historical anchor frames, oldest first */
   int64_t first_frame = -1, last_frame = -1, last_registration = -1;
   int64_t evicted_total = 0;
@@ -235,6 +254,7 @@ extern "C" orc_state* orc_create(const orc_config* cfg) {
   } else if (cfg->grid_h < 1 || cfg->grid_w < 1 || cfg->anchor_tokens > cfg->grid_h * cfg->grid_w) {
     return nullptr;
   }
+  if (cfg->camera_cache && cfg->score_mode == ORC_SCORE_QK) return nullptr; /* the probe concerns the aggregator */
   const int64_t M = cfg->n_special + (int64_t)cfg->grid_h * cfg->grid_w;
   /* Eq. 9: the protected set can reach M + K_max * A; the budget must hold it.  (Camera cache: an anchor is the
    * frame's one token.) */
@@ -285,6 +305,7 @@ extern "C" int orc_attend(orc_state* st, int64_t frame_id, const float* q, const
   }
   st->k.insert(st->k.end(), k, k + (size_t)M * C);
   st->v.insert(st->v.end(), v, v + (size_t)M * C);
+  if (st->cfg.score_mode == ORC_SCORE_QK) st->q_frame.assign(q, q + (size_t)M * C);
   if (st->first_frame < 0) {
     st->first_frame = frame_id;
     st->last_registration = frame_id; /* the first frame is the initial anchor */
@@ -338,7 +359,10 @@ extern "C" int orc_compress(orc_state* st, const float* resid, const float* conf
 
   /* Activation Value Rating (Eq. 5) and smoothing (Eq. 6) of the new frame. */
   std::vector<double> s(M), s_smooth(M);
-  orc_residual_norms(resid, M, C, s.data());
+  if (cfg.score_mode == ORC_SCORE_QK) /* Supp. D: the frame's queries against its own keys instead of Eq. 5 */
+    orc_qk_scores(st->q_frame.data(), &st->k[(size_t)n * C], M, cfg.n_heads, cfg.head_dim, s.data());
+  else
+    orc_residual_norms(resid, M, C, s.data());
   orc_smooth(s.data(), cfg.n_special, cfg.grid_h, cfg.grid_w, cfg.alpha, s_smooth.data());
   for (int32_t j = 0; j < M; ++j) st->stored[n + j] = (float)s_smooth[j];
 
@@ -367,7 +391,7 @@ extern "C" int orc_compress(orc_state* st, const float* resid, const float* conf
 
   /* Priorities (Eq. 7), or the stored-residual reading. */
   std::vector<float> r(N);
-  if (cfg.score_mode == ORC_SCORE_HYBRID) {
+  if (cfg.score_mode == ORC_SCORE_HYBRID || cfg.score_mode == ORC_SCORE_QK) {
     std::vector<double> d(std::max(n, 1));
     orc_diversity(st->k.data(), n, C, cfg.n_heads, cfg.diversity_per_head, d.data());
     orc_hybrid(d.data(), s_smooth.data(), st->flags.data(), n, M, cfg.beta, r.data());

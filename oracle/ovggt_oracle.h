@@ -32,7 +32,7 @@ extern "C" {
 #endif
 
 enum { ORC_FLAG_EVICTABLE = 0, ORC_FLAG_INIT = 1, ORC_FLAG_HIST = 2 };
-enum { ORC_SCORE_HYBRID = 0, ORC_SCORE_RESIDUAL_STORED = 1, ORC_SCORE_RANDOM = 2 };
+enum { ORC_SCORE_HYBRID = 0, ORC_SCORE_RESIDUAL_STORED = 1, ORC_SCORE_RANDOM = 2, ORC_SCORE_QK = 3 };
 
 typedef struct {
   int32_t n_heads, head_dim;             /* C = n_heads * head_dim */
@@ -54,6 +54,14 @@ typedef struct orc_state orc_state;
 
 /* Eq. 5: s_j = || r_j ||_2 for the M rows of R [M, C]. */
 void orc_residual_norms(const float* R, int32_t M, int32_t C, double* s);
+
+/* The query-key baseline of the scoring probe (Supp. D): the current-frame criterion is replaced by a dot product
+ * of queries and keys that needs no attention matrix.  The paper gives no formula; the reading taken here is the
+ * mean, over the frame's M queries and the heads, of the scaled attention logit that new token j receives:
+ *   s_j = 1 / (M * n_heads) * sum_h sum_i  (q_{i,h} . k_{j,h}) / sqrt(head_dim),
+ * Q, K [M, C] being the frame's own queries and keys.  Everything after the criterion (Eq. 6, Eq. 7 with the key
+ * diversity of the cached rows, Eq. 8) is as in the hybrid mode; the residual is not used. */
+void orc_qk_scores(const float* Q, const float* K, int32_t M, int32_t n_heads, int32_t head_dim, double* s);
 
 /* Eq. 6: patch part of s (after the first n_special entries) as a grid_h x grid_w
  * map, smoothed with a 3x3 Gaussian (sigma = 1, replicate border); aux tokens copied. */

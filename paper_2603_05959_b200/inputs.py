@@ -27,6 +27,7 @@ DTYPE_BF16 = 1
 SCORE_HYBRID = 0
 SCORE_RESIDUAL_STORED = 1
 SCORE_RANDOM = 2
+SCORE_QK = 3
 
 
 @dataclasses.dataclass(frozen=True)

@@ -485,6 +485,62 @@ def test_random_eviction_mode_keeps_a_uniform_subset_and_every_protected_row():
     assert len(evicted_pos) > 1500 and hist[1:].min() > 0.15
 
 
+# ------------------------------------------------------------------ Supp. D: the query-key criterion
+
+def test_qk_scores_are_the_mean_scaled_logits_a_key_receives():
+    """Against the library's batched matmul: the logits softmax would see, averaged over queries and heads; and the
+    closed form through the mean query.  M, H, d all differ and Q is not K, so a transposed operand, a sum over the
+    wrong axis or a missing 1/sqrt(d) fails."""
+    rng = np.random.default_rng(11)
+    M, H, d = 13, 3, 8
+    Q = rng.standard_normal((M, H * d)).astype(np.float32) + 0.3
+    K = rng.standard_normal((M, H * d)).astype(np.float32) - 0.2
+    got = orc.qk_scores(Q, K, H)
+    q = torch.from_numpy(Q).double().view(M, H, d).transpose(0, 1)      # [H, M, d]
+    k = torch.from_numpy(K).double().view(M, H, d).transpose(0, 1)
+    logits = torch.matmul(q, k.transpose(1, 2)) / math.sqrt(d)          # [H, i, j]
+    want = logits.mean(dim=(0, 1)).numpy()
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-13)
+    qbar = Q.astype(np.float64).mean(axis=0)                            # one C-vector
+    np.testing.assert_allclose(got, K.astype(np.float64) @ qbar / (H * math.sqrt(d)), rtol=1e-12, atol=1e-13)
+    assert np.abs(got - orc.qk_scores(K, Q, H)).max() > 1e-3             # queries and keys are not interchangeable
+    # a key that is the zero vector receives logit 0 from everyone; scaling the keys scales the scores
+    K2 = K.copy(); K2[4] = 0.0
+    assert orc.qk_scores(Q, K2, H)[4] == 0.0
+    np.testing.assert_allclose(orc.qk_scores(Q, 2.0 * K, H), 2.0 * got, rtol=1e-12)
+
+
+def test_qk_mode_replaces_only_the_current_frame_criterion():
+    """The stream in query-key mode: the new rows' priorities are beta x min-max of the smoothed query-key scores
+    (recomputed here with numpy and scipy), the cached rows' priorities equal those of the hybrid mode on the same
+    cache, and the residual plays no part."""
+    base = gen.config_tiny().replace(anchor_tokens=0, n_frames=8, budget=10_000)      # nothing is evicted: same caches
+    cfg = base.replace(score_mode=gen.SCORE_QK)
+    qk, hy = orc.OracleLayer.from_stream(cfg), orc.OracleLayer.from_stream(base)
+    M, H, d = cfg.tokens_per_frame, cfg.n_heads, cfg.head_dim
+    for t in range(cfg.n_frames):
+        fi = gen.frame_inputs(cfg, t)
+        qk.attend(t, fi.q, fi.k, fi.v, compute=False)
+        hy.attend(t, fi.q, fi.k, fi.v, compute=False)
+        out = qk.compress(None, fi.conf, fi.rho)
+        ref = hy.compress(fi.resid, fi.conf, fi.rho)
+        n = len(out["r"]) - M
+        if t == 0:
+            assert np.all(np.isinf(out["r"]))                                          # first frame: protected
+            continue
+        np.testing.assert_array_equal(out["r"][:n], ref["r"][:n])                      # (1 - beta) x diversity part
+        s = (fi.k.astype(np.float64) @ fi.q.astype(np.float64).mean(axis=0)) / (H * math.sqrt(d))
+        grid = s[cfg.n_special:].reshape(cfg.grid_h, cfg.grid_w)
+        g = np.exp(-0.5 * np.array([[2, 1, 2], [1, 0, 1], [2, 1, 2]], dtype=np.float64))
+        sm = s.copy()
+        sm[cfg.n_special:] = ((1 - cfg.alpha) * grid + cfg.alpha * scipy.ndimage.correlate(
+            grid, g / g.sum(), mode="nearest")).ravel()
+        want = cfg.beta * (sm - sm.min()) / (sm.max() - sm.min())
+        np.testing.assert_allclose(out["r"][n:], want, rtol=0, atol=2e-6)
+        assert np.abs(out["r"][n:] - ref["r"][n:]).max() > 0.05                        # not the residual criterion
+        np.testing.assert_allclose(qk.export(with_kv=False)["stored"][n:], sm, rtol=1e-6)
+
+
 # ------------------------------------------------------------------ Supp. C: the camera head's cache
 
 def _camera_token(cfg, t, tag):
