@@ -63,8 +63,15 @@ enum { OVGGT_DTYPE_F32 = 0, OVGGT_DTYPE_BF16 = 1 };
  * (Supp. A): the rows that leave are drawn uniformly at random under the same budget - every evictable row gets a
  * fresh uniform priority per step, the top 24 bits of SplitMix64(SplitMix64(random_seed ^ frame_id) + token_id)
  * scaled by 2^-24 (SplitMix64(x): z = x + 0x9E3779B97F4A7C15; z = (z ^ z >> 30) * 0xBF58476D1CE4E5B9;
- * z = (z ^ z >> 27) * 0x94D049BB133111EB; z ^ z >> 31), so that a run is reproducible from its seed. */
-enum { OVGGT_SCORE_HYBRID = 0, OVGGT_SCORE_RESIDUAL_STORED = 1, OVGGT_SCORE_RANDOM = 2 };
+ * z = (z ^ z >> 27) * 0x94D049BB133111EB; z ^ z >> 31), so that a run is reproducible from its seed.
+ * QK is the query-key baseline of the scoring probe (Supp. D): the hybrid mode with the residual norm of a new token
+ * (Eq. 5) replaced by a dot product of queries and keys that needs no attention matrix.  The paper prints no formula;
+ * the reading built here is the mean, over the frame's M queries and the heads, of the scaled logit new token j
+ * receives, s_j = 1 / (M n_heads) sum_h sum_i (q_{i,h} . k_{j,h}) / sqrt(head_dim), computed through the column sums
+ * of Q.  The attend half computes it from io->q and io->k and keeps it per layer until the layer's compress half,
+ * whose io->resid is then not read (it may be NULL); Eq. 6-8 and the key diversity of cached rows are unchanged.
+ * Not available for a camera-head cache. */
+enum { OVGGT_SCORE_HYBRID = 0, OVGGT_SCORE_RESIDUAL_STORED = 1, OVGGT_SCORE_RANDOM = 2, OVGGT_SCORE_QK = 3 };
 enum { OVGGT_FLAG_EVICTABLE = 0, OVGGT_FLAG_INIT = 1, OVGGT_FLAG_HIST = 2 };
 /* Where surviving K/V rows live after Eq. 8 (the paper fixes the survivor set, not a layout):
  *  FILL_HOLES     one K/V buffer per layer; the rows admitted from the new frame are copied into the slots the
@@ -101,7 +108,8 @@ typedef struct {
   const void* q;                /* [M, C] queries of the frame                     (attend) */
   const void* k;                /* [M, C] keys of the frame                        (attend) */
   const void* v;                /* [M, C] values of the frame                      (attend) */
-  const void* resid;            /* [M, C] FFN residual rows, LayerScale included   (compress, Eq. 5) */
+  const void* resid;            /* [M, C] FFN residual rows, LayerScale included   (compress, Eq. 5; unused and
+                                   optional in OVGGT_SCORE_QK) */
   const float* conf;            /* [grid_h*grid_w] per-patch confidence, or NULL = no anchor candidate (compress) */
   float rho;                    /* coverage ratio of the latest anchor in this view; NaN = no decision (compress) */
   const float* score_override;  /* [n + M] fp32 or NULL: priorities the selection ranks instead of its own (compress) */

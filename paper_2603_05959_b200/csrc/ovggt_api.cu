@@ -201,6 +201,21 @@ int launch_colsum(const void* K, int rows, int C, int dtype, float* part, float*
   return OVGGT_OK;
 }
 
+// Supp. D, query-key criterion: s[j] = mean over the M queries and the heads of q_i . k_j / sqrt(d), taken through
+// the column sums of Q (qsum [C] after part [colsum_parts(M), C]; three small kernels).
+int launch_qk_scores(const void* q, const void* k, int M, int C, int n_heads, int dtype, float* part, float* qsum,
+                     float* s, cudaStream_t st) {
+  int rc = launch_colsum(q, M, C, dtype, part, qsum, st);
+  if (rc) return rc;
+  const int nvec = C * elem_bytes(dtype) / 16;
+  const float scale = 1.0f / ((float)M * (float)n_heads * sqrtf((float)(C / n_heads)));
+  const int grid = (M + 7) / 8;
+  if (dtype == kBF16) k_row_dots<kBF16><<<grid, 256, 0, st>>>((const uint4*)k, M, nvec, qsum, scale, s);
+  else                k_row_dots<kF32><<<grid, 256, 0, st>>>((const uint4*)k, M, nvec, qsum, scale, s);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
 // The hole-filling move (and, with delta, what it does to the key column sums).
 int launch_fill_holes(void* kc, void* vc, const int* msrc, const int* mdst, const int* mj, const int* n_moves, int max_moves,
                       int C, int dtype, int* slot_meta, float* delta, cudaStream_t st, int rows_cap, int n_meta,
@@ -301,6 +316,7 @@ struct ovggt_cache {
   int64_t decided_demote = -1;
   // shared scratch
   float *colsum_part = nullptr, *ksum = nullptr;
+  float *qk_part = nullptr, *qk_sum = nullptr;       // OVGGT_SCORE_QK: column sums of the frame's queries
   void* attn_scratch = nullptr;
   int* status = nullptr;
   // two sets of staging buffers for ovggt_layer_step_host: the copies of one step overlap the kernels of the step before
@@ -378,8 +394,9 @@ bool config_ok(const ovggt_config* c, int* err) {
   if (c->k_max < 0 || c->k_max > OVGGT_MAX_ANCHORS || c->min_anchor_interval < 0) return false;
   if (c->dtype != kF32 && c->dtype != kBF16) return false;
   if (c->score_mode != OVGGT_SCORE_HYBRID && c->score_mode != OVGGT_SCORE_RESIDUAL_STORED &&
-      c->score_mode != OVGGT_SCORE_RANDOM)
+      c->score_mode != OVGGT_SCORE_RANDOM && c->score_mode != OVGGT_SCORE_QK)
     return false;
+  if (c->score_mode == OVGGT_SCORE_QK && c->camera_head) return false;   // the probe concerns the aggregator's caches
   if (c->compaction != OVGGT_COMPACT_FILL_HOLES && c->compaction != OVGGT_COMPACT_STABLE_GATHER) return false;
   if (!(c->alpha >= 0.0f && c->alpha <= 1.0f) || !(c->beta >= 0.0f && c->beta <= 1.0f)) return false;
   const int64_t M = c->n_special + (int64_t)c->grid_h * c->grid_w;
@@ -469,6 +486,8 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
   const size_t o_ksum = L.take(colsum_scratch_bytes(C));
   const size_t o_attn = L.take(ovggt_k_attention_scratch_bytes(M, max_rows, c->n_heads));
   const size_t o_status = L.take(64);
+  const bool qk = c->score_mode == OVGGT_SCORE_QK;
+  const size_t o_qk = qk ? L.take((size_t)(colsum_parts(M) + 1) * C * 4) : 0;
   size_t o_stage[2][5], o_conf[2];
   for (int p = 0; p < 2; ++p) {
     for (int i = 0; i < 5; ++i) o_stage[p][i] = L.take((size_t)M * C * eb);
@@ -479,6 +498,10 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
     h->ksum = reinterpret_cast<float*>(base + o_ksum);
     h->attn_scratch = base + o_attn;
     h->status = reinterpret_cast<int*>(base + o_status);
+    if (qk) {
+      h->qk_part = reinterpret_cast<float*>(base + o_qk);
+      h->qk_sum = h->qk_part + (size_t)colsum_parts(M) * C;
+    }
     for (int p = 0; p < 2; ++p) {
       h->stage_q[p] = base + o_stage[p][0];
       h->stage_k[p] = base + o_stage[p][1];
@@ -491,6 +514,10 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
   }
   return align_up(L.total, 1024);
 }
+
+// Score modes whose cached rows are ranked by key diversity (Eq. 7); the query-key probe (Supp. D) differs from the
+// hybrid mode only in the criterion of the new frame's rows.
+bool ranks_by_diversity(int mode) { return mode == OVGGT_SCORE_HYBRID || mode == OVGGT_SCORE_QK; }
 
 int check_layer(ovggt_cache* h, int32_t layer) {
   if (!h) return OVGGT_ERR_INVALID_ARG;
@@ -706,17 +733,28 @@ int enqueue_attention(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, c
   return OVGGT_OK;
 }
 
+// Query-key mode (Supp. D): the criterion of the new frame's rows, from the frame's own q and k; kept in the layer's
+// s_raw until the layer's compress.
+int enqueue_qk_scores(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io, cudaStream_t st) {
+  if (h->cfg.score_mode != OVGGT_SCORE_QK) return OVGGT_OK;
+  ProfScope ps(h, OVGGT_PROF_ROW_NORMS, st);
+  return launch_qk_scores(io->q, io->k, h->M, h->C, h->cfg.n_heads, h->cfg.dtype, h->qk_part, h->qk_sum, S.s_raw, st);
+}
+
 // Eq. 5 and the diversity score of Sec. 3.2 for the frame io describes: everything the selection needs that does not
 // depend on the anchor decision.  Reads the cached keys [0, n) and the frame's residual, so it may run before the
 // frame's K/V are appended.
 int enqueue_scores(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io, cudaStream_t st) {
   const ovggt_config& c = h->cfg;
   const int M = h->M, C = h->C, n = S.n, kb = S.kv;
-  const bool hybrid = c.score_mode == OVGGT_SCORE_HYBRID && n > 0;
+  const bool hybrid = ranks_by_diversity(c.score_mode) && n > 0;
+  // query-key mode: s_raw was written by the attend half (enqueue_qk_scores); the residual is not read
+  const void* resid = c.score_mode == OVGGT_SCORE_QK ? nullptr : io->resid;
   int rc = OVGGT_OK;
   if (!hybrid) {
+    if (!resid) return OVGGT_OK;
     ProfScope ps(h, OVGGT_PROF_ROW_NORMS, st);
-    return launch_row_norms(io->resid, M, C, c.dtype, S.s_raw, st);
+    return launch_row_norms(resid, M, C, c.dtype, S.s_raw, st);
   }
   if (fill_layout(h)) {
     // Column sums of the cached keys: continued from the last step's sums and the corrections its move left, or
@@ -732,16 +770,16 @@ int enqueue_scores(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io, cuda
       S.since_refresh += 1;
     }
     return launch_diversity_sliced(S.kbuf[kb], n, C, c.dtype, S.ksum[S.kcur], fresh ? 1 : 1 + kFillSlices,
-                                   S.ksum[S.kcur ^ 1], S.d, io->resid, M, S.s_raw, st);
+                                   S.ksum[S.kcur ^ 1], S.d, resid, M, S.s_raw, st);
   }
   if (S.colsum_nparts > 0) {   // stable layout, sums left by the last compaction
     ProfScope ps(h, OVGGT_PROF_DIVERSITY, st);
     return launch_diversity_from_parts(S.kbuf[kb], n, C, c.dtype, S.colsum_part, S.colsum_nparts, h->ksum, S.d,
-                                       io->resid, M, S.s_raw, st);
+                                       resid, M, S.s_raw, st);
   }
-  {
+  if (resid) {
     ProfScope ps(h, OVGGT_PROF_ROW_NORMS, st);
-    rc = launch_row_norms(io->resid, M, C, c.dtype, S.s_raw, st);
+    rc = launch_row_norms(resid, M, C, c.dtype, S.s_raw, st);
   }
   if (rc) return rc;
   ProfScope ps(h, OVGGT_PROF_DIVERSITY, st);
@@ -756,9 +794,12 @@ struct MirroredDecision { bool registered; int64_t demoted_frame; };
 int validate_compress(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, const MirroredDecision* mirrored) {
   int rc = check_layer(h, layer);
   if (rc) return rc;
-  if (!io || !io->resid) return OVGGT_ERR_INVALID_ARG;
+  if (!io) return OVGGT_ERR_INVALID_ARG;
   if ((h->cfg.camera_head != 0) != (mirrored != nullptr)) return OVGGT_ERR_INVALID_ARG;
-  if (!aligned16(io->resid)) return OVGGT_ERR_MISALIGNED;
+  if (h->cfg.score_mode != OVGGT_SCORE_QK) {   // (query-key mode does not read the residual)
+    if (!io->resid) return OVGGT_ERR_INVALID_ARG;
+    if (!aligned16(io->resid)) return OVGGT_ERR_MISALIGNED;
+  }
   const LayerState& S = h->layers[layer];
   if (!S.pending || io->frame_id != S.pending_frame) return OVGGT_ERR_FRAME_ORDER;
   const int N = S.n + h->M, ncta = select_cluster_ctas(N);
@@ -814,7 +855,7 @@ CompressParams select_params(ovggt_cache* h, LayerState& S, const ovggt_frame_io
   P.n_special = c.n_special; P.grid_h = c.grid_h; P.grid_w = c.grid_w;
   P.alpha = c.alpha; P.w_center = h->w_center; P.w_edge = h->w_edge; P.w_corner = h->w_corner;
   P.beta = c.beta;
-  P.mode = c.score_mode;
+  P.mode = c.score_mode == OVGGT_SCORE_QK ? OVGGT_SCORE_HYBRID : c.score_mode;   // same Eq. 6-8, other s_raw
   P.protect_new = (first && c.protect_first_frame) ? OVGGT_FLAG_INIT
                                                    : ((c.camera_head && h->decided_register) ? OVGGT_FLAG_HIST : 0);
   P.lone_new = c.camera_head ? 1.0f : -1.0f;
@@ -855,7 +896,7 @@ void close_compress(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io) {
 // step's diversity launch used and wrote to ksum[kcur ^ 1], and describe the next cache only if every slot below B
 // held a cached row (n == B: steady state).
 bool move_leaves_corrections(const ovggt_cache* h, const LayerState& S) {
-  return h->cfg.score_mode == OVGGT_SCORE_HYBRID && h->C * h->elem / 16 <= kCompactSumMaxVec && S.n == S.budget;
+  return ranks_by_diversity(h->cfg.score_mode) && h->C * h->elem / 16 <= kCompactSumMaxVec && S.n == S.budget;
 }
 
 // The compress half on stream st.  The stable gather writes another buffer, so the whole half may run beside an
@@ -904,7 +945,7 @@ int compress_impl(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, cudaS
     }
   } else {
     ProfScope ps(h, OVGGT_PROF_COMPACT, st_move);
-    const bool fuse = c.score_mode == OVGGT_SCORE_HYBRID && C * h->elem / 16 <= kCompactSumMaxVec;
+    const bool fuse = ranks_by_diversity(c.score_mode) && C * h->elem / 16 <= kCompactSumMaxVec;
     S.colsum_nparts = 0;
     if (fuse)
       rc = launch_compact_colsum(S.kbuf[kb], S.vbuf[kb], S.surv, n_keep, C, c.dtype, S.kbuf[kb ^ 1], S.vbuf[kb ^ 1],
@@ -950,10 +991,11 @@ int compress_all_layers(ovggt_cache* h, const ovggt_frame_io* ios, cudaStream_t 
       for (int i = 0; i < cnt; ++i) {
         LayerState& S = h->layers[l0 + i];
         S.scores_frame = -1;
-        const bool hybrid = c.score_mode == OVGGT_SCORE_HYBRID && S.n > 0;
+        const bool hybrid = ranks_by_diversity(c.score_mode) && S.n > 0;
         DiversityArgs& A = db.a[i];
         A = DiversityArgs{};
-        A.resid = (const uint4*)ios[l0 + i].resid; A.resid_rows = M; A.s_raw = S.s_raw;
+        A.resid = c.score_mode == OVGGT_SCORE_QK ? nullptr : (const uint4*)ios[l0 + i].resid;
+        A.resid_rows = M; A.s_raw = S.s_raw;
         if (hybrid) {
           const bool fresh = !S.ksum_valid || S.since_refresh >= kColsumRefreshEvery;
           if (fresh) {
@@ -1012,7 +1054,9 @@ extern "C" int ovggt_layer_attend(ovggt_cache* h, int32_t layer, const ovggt_fra
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc = enqueue_append(h, layer, io, st);
   if (rc) return rc;
-  return enqueue_attention(h, layer, io, st);
+  rc = enqueue_attention(h, layer, io, st);
+  if (rc) return rc;
+  return enqueue_qk_scores(h, h->layers[layer], io, st);
 }
 
 extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
@@ -1047,8 +1091,9 @@ extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame
   if (rc) return rc;
   if (h->cfg.camera_head) return OVGGT_ERR_INVALID_ARG;   // the camera head's cache needs the aggregator's decision
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const bool can_overlap = h->side && h->overlap && io && io->resid && aligned16(io->resid) && io->q && io->k &&
-                           io->v && io->out && !h->layers[layer].pending;
+  const bool resid_ok = io && (h->cfg.score_mode == OVGGT_SCORE_QK || (io->resid && aligned16(io->resid)));
+  const bool can_overlap = h->side && h->overlap && resid_ok && io->q && io->k && io->v && io->out &&
+                           !h->layers[layer].pending;
   if (!can_overlap) {
     rc = ovggt_layer_attend(h, layer, io, stream);
     if (rc) return rc;
@@ -1067,7 +1112,8 @@ extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame
   if (rc) return rc;
   CK(cudaEventRecord(h->ev_fork, st));
   CK(cudaStreamWaitEvent(h->side, h->ev_fork, 0));
-  rc = enqueue_scores(h, S, io, h->side);
+  rc = enqueue_qk_scores(h, S, io, h->side);
+  if (rc == OVGGT_OK) rc = enqueue_scores(h, S, io, h->side);
   if (rc == OVGGT_OK) {
     S.scores_frame = io->frame_id;
     rc = enqueue_attention(h, layer, io, st);

@@ -40,6 +40,29 @@ __global__ void __launch_bounds__(256) k_row_norms(const uint4* __restrict__ x, 
   if (row < rows) warp_row_norm<DT>(x, row, nvec, s);
 }
 
+// out[row] = scale * sum_c x[row, c] * vec[c]; one warp per row, the same order of accumulation as warp_row_norm.
+// With vec = the column sums of the frame's queries and scale = 1 / (M H sqrt(d)) this is the query-key criterion of
+// the scoring probe (Supp. D): the mean scaled logit the key of row `row` receives from the M queries over all heads.
+template <int DT>
+__global__ void __launch_bounds__(256) k_row_dots(const uint4* __restrict__ x, int rows, int nvec,
+                                                  const float* __restrict__ vec, float scale, float* __restrict__ out) {
+  constexpr int VEC = VecOf<DT>::n;
+  const int row = (int)((blockIdx.x * (unsigned)blockDim.x + threadIdx.x) >> 5);
+  if (row >= rows) return;                       // whole warps leave together: a row belongs to one warp
+  const int lane = threadIdx.x & 31;
+  const uint4* p = x + (size_t)row * nvec;
+  float acc = 0.0f;
+  for (int v = lane; v < nvec; v += 32) {
+    float f[VEC];
+    unpack<DT>(ld_nc(p + v), f);
+    const float* w = vec + (size_t)v * VEC;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc = __fmaf_rn(f[e], __ldg(w + e), acc);
+  }
+  acc = warp_sum(acc);
+  if (lane == 0) out[row] = acc * scale;
+}
+
 // Column sums of K [rows, C], stage 1: CTA p sums its contiguous chunk of rows, in row order,
 // into part[p, C].  Thread t owns vector columns t, t + blockDim, ...
 template <int DT>
