@@ -454,7 +454,10 @@ def run_c2(args) -> None:
             "roofline": {"kernel": "k_attn_tcgen05", "bound": "tensor", "achieved": achieved,
                          "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                          "peak_kind": f"{peak_kind} burst cuBLAS bf16 peak", "traffic": attention_traffic(),
-                         "algorithmic_flops": attn_flops, "launch_ms": attn_ms},
+                         "algorithmic_flops": attn_flops, "launch_ms": attn_ms,
+                         # the launch is timed right after the K timed steps, at the clocks the step itself ran at;
+                         # the same figure against the sustained (power-capped) cuBLAS peak, for long runs
+                         "frac_of_sustained_peak": achieved / float(peaks["bf16_tflops_sustained"])},
             "kernels": kernels,
             "ms_per_frame": flatness(per_step),
             "single_stream_l2_resident": None if single_ms is None else

@@ -101,7 +101,7 @@ __device__ inline int block_sum_int(int x, int* sh) {
 }
 
 // Exclusive prefix sum of x over the threads of the block in thread order; *total = block sum.
-__device__ inline int block_excl_scan_int(int x, int* sh, int* total) {
+__device__ __noinline__ int block_excl_scan_int(int x, int* sh, int* total) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
   int incl = x;
 #pragma unroll
@@ -121,7 +121,7 @@ __device__ inline int block_excl_scan_int(int x, int* sh, int* total) {
   return base + incl - x;
 }
 
-__device__ inline void block_minmax(float lo, float hi, float* sh, float* out_lo, float* out_hi) {
+__device__ __noinline__ void block_minmax(float lo, float hi, float* sh, float* out_lo, float* out_hi) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {

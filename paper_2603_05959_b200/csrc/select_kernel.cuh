@@ -43,7 +43,7 @@ __device__ __forceinline__ void cta_range(int N, int ncta, int rank, int* begin,
 }
 
 // Warp 0 finds the digit whose bin holds the krem-th largest remaining key, given bin counts tot[256].
-__device__ __forceinline__ void find_digit(const int* tot, int krem, SelectShared* sh) {
+__device__ __noinline__ void find_digit(const int* tot, int krem, SelectShared* sh) {
   const int tid = threadIdx.x;
   if (tid < 32) {
     int c[8], local = 0;
@@ -72,7 +72,7 @@ __device__ __forceinline__ void find_digit(const int* tot, int krem, SelectShare
 
 // Digit histogram of the keys that match (mask, prefix).  Keys of one step share their leading bits, so lanes
 // of a warp mostly hit the same bin: lanes with equal digits are grouped and one of them adds the group's count.
-__device__ __forceinline__ void digit_histogram(const uint32_t* keys, int cnt, uint32_t mask, uint32_t prefix,
+__device__ __noinline__ void digit_histogram(const uint32_t* keys, int cnt, uint32_t mask, uint32_t prefix,
                                                 int shift, int* hist) {
   const int tid = threadIdx.x, nthr = blockDim.x;
   for (int i0 = 0; i0 < cnt; i0 += nthr) {
@@ -103,6 +103,7 @@ __device__ inline int cluster_select(cg::cluster_group& cluster, const uint32_t*
     uint32_t prefix = 0, mask = 0;
     int krem = B;
     int buf = 0;
+#pragma unroll 1
     for (int shift = 24; shift >= 0; shift -= 8, buf ^= 1) {
       int* hist = sh->hist[buf];
       for (int b = tid; b < 256; b += nthr) hist[b] = 0;
@@ -111,8 +112,13 @@ __device__ inline int cluster_select(cg::cluster_group& cluster, const uint32_t*
       cluster.sync();
       // every CTA folds all histograms and finds the same digit
       if (tid < 256) {
+        int v[kSelectMaxCtas];
+#pragma unroll
+        for (int r = 0; r < kSelectMaxCtas; ++r)      // all remote loads in flight before the first add
+          v[r] = r < ncta ? cluster.map_shared_rank(hist, r)[tid] : 0;
         int t = 0;
-        for (int r = 0; r < ncta; ++r) t += cluster.map_shared_rank(hist, r)[tid];
+#pragma unroll
+        for (int r = 0; r < kSelectMaxCtas; ++r) t += v[r];
         sh->tot[tid] = t;
       }
       __syncthreads();
@@ -198,6 +204,7 @@ __device__ inline void block_top_mark(const uint32_t* keys, uint8_t* keep, int c
   if (!keep_all && A > 0) {
     uint32_t prefix = 0, mask = 0;
     int krem = A;
+#pragma unroll 1
     for (int shift = 24; shift >= 0; shift -= 8) {
       for (int b = tid; b < 256; b += nthr) sh->tot[b] = 0;
       __syncthreads();
