@@ -3,21 +3,26 @@
 // One CTA owns one 128-row query tile of one head and a contiguous range of 192-row KV tiles.  Each KV
 // tile is processed as two 96-row halves with their own S buffer in tensor memory, so the MMAs of one half
 // run while the softmax warps work on the other and the softmax never waits for a whole QK^T -> PV chain.
-//   warps 0-3   softmax: one thread per query row reads its 96 S values of a half with tcgen05.ld, keeps a
-//               running reference maximum (rescaling O only when the maximum grows by more than 2^8; the maximum
-//               is gathered inside the exponential pass, and the pass is repeated in the rare case that it outgrew
-//               the reference), takes one pair of exponentials in four on the FMA pipes, writes P as bf16 over the
-//               first 48 columns of that half, and at the end normalises and stores O
+//   warps 0-3   softmax: one thread per query row reads its 96 S values of a half with tcgen05.ld and turns them into
+//               p = 2^(s c - reference).  Where the cache supplies a bound of the key norms, the reference is fixed
+//               once (the bound of this row's logits, moved a whole number of powers of two above the first half's
+//               maximum): nothing is tracked and O is never rescaled.  Without a bound the reference is a running
+//               maximum, gathered inside the exponential pass, and O is rescaled only when it grows by more than 2^8
+//               (the pass is then repeated).  One pair of exponentials in three is a cubic on the FMA pipes, the rest
+//               go to the special-function unit; P is written as bf16 over the first 48 columns of that half; at
+//               the end the warps normalise and store O (or the split's partial O, maximum and sum)
 //   warp 4      TMA producer: Q once, then K and V tiles into 128-byte-swizzled shared-memory stages
 //   warp 5      allocates tensor memory and issues tcgen05.mma:  S_h = Q K_h^T  (SS, fp32 in TMEM),
 //               O += P_h V_h (P read from TMEM as the A operand, V MN-major from shared memory); the whole warp
 //               walks the loop so that descriptors stay warp-uniform, one elected lane issues
 //   warps 6-7   only complete the second warpgroup, which hands its registers to the softmax warpgroup
 // With head_dim 64 a 128 x 128 tile needs 512 tensor-pipe cycles but 1024 cycles of the 16-per-clock
-// exponential unit, so the softmax rounds bound the kernel; two CTAs are resident per SM (256 TMEM columns and
-// ~115 KB shared memory each) to keep that unit fed from two independent query tiles.  The KV range may be split
-// across CTAs; partial (O, max, sum) triples are merged by a second kernel.  Every mbarrier wait is bounded: on
-// expiry the CTA records OVGGT_ERR_TIMEOUT in the status word and leaves through the common teardown.
+// exponential unit, so the softmax rounds bound the kernel (a 96-column round is about 1,700 cycles, 1,200 of them
+// the exponential pass, whose instruction mix tops out near 0.15 columns per cycle per scheduler); two CTAs are
+// resident per SM (256 TMEM columns and ~115 KB shared memory each) to keep that unit fed from two independent query
+// tiles.  The KV range may be split across CTAs; partial (O, max, sum) triples are merged by a second kernel.  Every
+// mbarrier wait is bounded: on expiry the CTA records OVGGT_ERR_TIMEOUT in the status word and leaves through the
+// common teardown.
 #pragma once
 
 #include <cuda.h>
