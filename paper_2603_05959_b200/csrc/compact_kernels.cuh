@@ -211,6 +211,7 @@ __global__ void __launch_bounds__(256) k_append(const uint4* __restrict__ k_new,
 // result does not depend on timing.  Requires nvec <= kCompactSumMaxVec when delta is asked for.
 constexpr int kFillSlices = 16;
 constexpr int kFillClusterCtas = 8;
+static_assert(kFillClusterCtas <= 8, "the cluster folds below read eight ranks at most");
 constexpr int kFillThreads = 256;
 
 struct FillArgs {
@@ -306,8 +307,12 @@ __device__ __forceinline__ void fill_holes_body(const FillArgs& A, int nvec) {
   const int cid = (int)blockIdx.x / ncta;
   for (int c = rank * 32 + (threadIdx.x & 31) + (threadIdx.x >> 5) * 32 * ncta; c < C;
        c += 32 * ncta * (blockDim.x >> 5)) {
+    float v[8];                                   // all remote reads in flight before the first add (clusters of <= 8)
+#pragma unroll
+    for (int q = 0; q < 8; ++q) v[q] = q < ncta ? cluster.map_shared_rank(cta_part, q)[c] : 0.0f;
     float t = 0.0f;
-    for (int q = 0; q < ncta; ++q) t += cluster.map_shared_rank(cta_part, q)[c];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) t += v[q];        // rank order
     delta[(size_t)cid * C + c] = t;
   }
   cluster.sync();   // no CTA may exit while others still read its shared memory
@@ -465,8 +470,12 @@ __global__ void __launch_bounds__(kAppendFillThreads) k_append_fill(const __grid
   const int cid = (int)blockIdx.x / ncta;
   for (int c = rank * 32 + (threadIdx.x & 31) + (threadIdx.x >> 5) * 32 * ncta; c < C;
        c += 32 * ncta * (blockDim.x >> 5)) {
+    float v[8];                                   // all remote reads in flight before the first add (clusters of <= 8)
+#pragma unroll
+    for (int q = 0; q < 8; ++q) v[q] = q < ncta ? cluster.map_shared_rank(cta_part, q)[c] : 0.0f;
     float t = 0.0f;
-    for (int q = 0; q < ncta; ++q) t += cluster.map_shared_rank(cta_part, q)[c];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) t += v[q];        // rank order, as a loop over the ranks would add them
     A.delta[(size_t)cid * C + c] = t;
   }
   cluster.sync();   // no CTA may exit while others still read its shared memory
