@@ -25,7 +25,7 @@ class OrcConfig(C.Structure):
     ]
 
 
-SCORE_HYBRID, SCORE_RESIDUAL_STORED, SCORE_RANDOM, SCORE_QK = 0, 1, 2, 3
+SCORE_HYBRID, SCORE_RESIDUAL_STORED, SCORE_RANDOM, SCORE_QK, SCORE_ATTN = 0, 1, 2, 3, 4
 
 
 def _f32(a):
@@ -65,6 +65,8 @@ def lib():
         L.orc_residual_norms.argtypes = [C.POINTER(C.c_float), C.c_int32, C.c_int32, C.POINTER(C.c_double)]
         L.orc_qk_scores.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_int32, C.c_int32, C.c_int32,
                                     C.POINTER(C.c_double)]
+        L.orc_attention_received.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_float), C.c_int32, C.c_int32,
+                                             C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_double)]
         L.orc_smooth.argtypes = [C.POINTER(C.c_double), C.c_int32, C.c_int32, C.c_int32, C.c_double,
                                  C.POINTER(C.c_double)]
         L.orc_diversity.argtypes = [C.POINTER(C.c_float), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
@@ -111,6 +113,16 @@ def qk_scores(Q: np.ndarray, K: np.ndarray, n_heads: int) -> np.ndarray:
     s = np.empty(Q.shape[0], dtype=np.float64)
     lib().orc_qk_scores(_ptr(Q, C.c_float), _ptr(K, C.c_float), Q.shape[0], n_heads, Q.shape[1] // n_heads,
                         _ptr(s, C.c_double))
+    return s
+
+
+def attention_received(Q: np.ndarray, K: np.ndarray, n_heads: int, first_col: int = 0, n_cols: int = -1) -> np.ndarray:
+    """Supp. D, attention-weight criterion: mean over queries and heads of the columns of softmax(Q K^T / sqrt(d))."""
+    Q, K = _f32(Q), _f32(K)
+    n_cols = K.shape[0] - first_col if n_cols < 0 else n_cols
+    s = np.empty(n_cols, dtype=np.float64)
+    lib().orc_attention_received(_ptr(Q, C.c_float), _ptr(K, C.c_float), Q.shape[0], K.shape[0], n_heads,
+                                 Q.shape[1] // n_heads, first_col, n_cols, _ptr(s, C.c_double))
     return s
 
 
@@ -255,8 +267,8 @@ class OracleLayer:
         return out
 
     def compress(self, resid, conf=None, rho=float("nan"), score_override=None):
-        if resid is None:   # SCORE_QK reads the queries kept by attend() instead
-            assert self.cfg.score_mode == SCORE_QK
+        if resid is None:   # these modes score the frame from what attend() kept
+            assert self.cfg.score_mode in (SCORE_QK, SCORE_ATTN)
         else:
             resid = _f32(resid)
             assert resid.shape == (self.M, self.C)

@@ -229,6 +229,34 @@ extern "C" void orc_attention(const float* Q, const float* K, const float* V, in
   }
 }
 
+/* ------------------------------------------------------------------ Supp. D, attention-weight criterion */
+extern "C" void orc_attention_received(const float* Q, const float* K, int32_t M, int32_t N, int32_t n_heads,
+                                       int32_t head_dim, int32_t first_col, int32_t n_cols, double* s) {
+  const int32_t C = n_heads * head_dim;
+  const double scale = 1.0 / std::sqrt((double)head_dim);
+  for (int32_t j = 0; j < n_cols; ++j) s[j] = 0.0;
+  std::vector<double> p(N);
+  for (int32_t h = 0; h < n_heads; ++h)
+    for (int32_t i = 0; i < M; ++i) {
+      /* row i of P_h, written out */
+      double mx = -std::numeric_limits<double>::infinity();
+      for (int32_t n = 0; n < N; ++n) {
+        double acc = 0.0;
+        for (int32_t c = 0; c < head_dim; ++c)
+          acc += (double)Q[(size_t)i * C + h * head_dim + c] * (double)K[(size_t)n * C + h * head_dim + c];
+        p[n] = acc * scale;
+        mx = std::max(mx, p[n]);
+      }
+      double denom = 0.0;
+      for (int32_t n = 0; n < N; ++n) {
+        p[n] = std::exp(p[n] - mx);
+        denom += p[n];
+      }
+      for (int32_t j = 0; j < n_cols; ++j) s[j] += p[first_col + j] / denom;
+    }
+  for (int32_t j = 0; j < n_cols; ++j) s[j] /= (double)M * (double)n_heads;
+}
+
 /* ------------------------------------------------------------------ state */
 struct orc_state {
   orc_config cfg;
@@ -238,6 +266,7 @@ struct orc_state {
   std::vector<float> stored;   /* smoothed activation score each row had when it was new */
   std::vector<float> k, v;     /* [rows, C] */
   std::vector<float> q_frame;  /* [M, C] queries of the pending frame (ORC_SCORE_QK only) */
+  std::vector<double> received; /* [M] attention the pending frame's tokens receive (ORC_SCORE_ATTN only) */
   std::deque<int64_t> anchors; /* active historical anchor frames, oldest first */
   int64_t first_frame = -1, last_frame = -1, last_registration = -1;
   int64_t evicted_total = 0;
@@ -254,7 +283,8 @@ extern "C" orc_state* orc_create(const orc_config* cfg) {
   } else if (cfg->grid_h < 1 || cfg->grid_w < 1 || cfg->anchor_tokens > cfg->grid_h * cfg->grid_w) {
     return nullptr;
   }
-  if (cfg->camera_cache && cfg->score_mode == ORC_SCORE_QK) return nullptr; /* the probe concerns the aggregator */
+  if (cfg->camera_cache && (cfg->score_mode == ORC_SCORE_QK || cfg->score_mode == ORC_SCORE_ATTN))
+    return nullptr; /* the probe concerns the aggregator */
   const int64_t M = cfg->n_special + (int64_t)cfg->grid_h * cfg->grid_w;
   /* Eq. 9: the protected set can reach M + K_max * A; the budget must hold it.  (Camera cache: an anchor is the
    * frame's one token.) */
@@ -306,6 +336,11 @@ extern "C" int orc_attend(orc_state* st, int64_t frame_id, const float* q, const
   st->k.insert(st->k.end(), k, k + (size_t)M * C);
   st->v.insert(st->v.end(), v, v + (size_t)M * C);
   if (st->cfg.score_mode == ORC_SCORE_QK) st->q_frame.assign(q, q + (size_t)M * C);
+  if (st->cfg.score_mode == ORC_SCORE_ATTN) { /* columns of the frame's own tokens in this very attention */
+    const int32_t N = (int32_t)st->ids.size();
+    st->received.assign(M, 0.0);
+    orc_attention_received(q, st->k.data(), M, N, st->cfg.n_heads, st->cfg.head_dim, N - M, M, st->received.data());
+  }
   if (st->first_frame < 0) {
     st->first_frame = frame_id;
     st->last_registration = frame_id; /* the first frame is the initial anchor */
@@ -361,6 +396,8 @@ extern "C" int orc_compress(orc_state* st, const float* resid, const float* conf
   std::vector<double> s(M), s_smooth(M);
   if (cfg.score_mode == ORC_SCORE_QK) /* Supp. D: the frame's queries against its own keys instead of Eq. 5 */
     orc_qk_scores(st->q_frame.data(), &st->k[(size_t)n * C], M, cfg.n_heads, cfg.head_dim, s.data());
+  else if (cfg.score_mode == ORC_SCORE_ATTN) /* Supp. D: the attention the new tokens received */
+    s = st->received;
   else
     orc_residual_norms(resid, M, C, s.data());
   orc_smooth(s.data(), cfg.n_special, cfg.grid_h, cfg.grid_w, cfg.alpha, s_smooth.data());
@@ -391,7 +428,7 @@ extern "C" int orc_compress(orc_state* st, const float* resid, const float* conf
 
   /* Priorities (Eq. 7), or the stored-residual reading. */
   std::vector<float> r(N);
-  if (cfg.score_mode == ORC_SCORE_HYBRID || cfg.score_mode == ORC_SCORE_QK) {
+  if (cfg.score_mode == ORC_SCORE_HYBRID || cfg.score_mode == ORC_SCORE_QK || cfg.score_mode == ORC_SCORE_ATTN) {
     std::vector<double> d(std::max(n, 1));
     orc_diversity(st->k.data(), n, C, cfg.n_heads, cfg.diversity_per_head, d.data());
     orc_hybrid(d.data(), s_smooth.data(), st->flags.data(), n, M, cfg.beta, r.data());

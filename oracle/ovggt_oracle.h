@@ -32,7 +32,7 @@ extern "C" {
 #endif
 
 enum { ORC_FLAG_EVICTABLE = 0, ORC_FLAG_INIT = 1, ORC_FLAG_HIST = 2 };
-enum { ORC_SCORE_HYBRID = 0, ORC_SCORE_RESIDUAL_STORED = 1, ORC_SCORE_RANDOM = 2, ORC_SCORE_QK = 3 };
+enum { ORC_SCORE_HYBRID = 0, ORC_SCORE_RESIDUAL_STORED = 1, ORC_SCORE_RANDOM = 2, ORC_SCORE_QK = 3, ORC_SCORE_ATTN = 4 };
 
 typedef struct {
   int32_t n_heads, head_dim;             /* C = n_heads * head_dim */
@@ -62,6 +62,14 @@ void orc_residual_norms(const float* R, int32_t M, int32_t C, double* s);
  * Q, K [M, C] being the frame's own queries and keys.  Everything after the criterion (Eq. 6, Eq. 7 with the key
  * diversity of the cached rows, Eq. 8) is as in the hybrid mode; the residual is not used. */
 void orc_qk_scores(const float* Q, const float* K, int32_t M, int32_t n_heads, int32_t head_dim, double* s);
+
+/* The attention-weight baseline of the scoring probe (Supp. D): the criterion that needs the materialised attention
+ * matrix.  Reading taken here (the paper prints no formula): the importance of a token is the attention it receives,
+ * averaged over the frame's M queries and the heads,
+ *   s_j = 1 / (M * n_heads) * sum_h sum_i P_h[i, first_col + j],   P_h = softmax(Q_h K_h^T / sqrt(head_dim)) over all N rows,
+ * for the n_cols columns from first_col on.  Q [M, C]; K [N, C].  (Over all N columns the s_j add up to 1.) */
+void orc_attention_received(const float* Q, const float* K, int32_t M, int32_t N, int32_t n_heads, int32_t head_dim,
+                            int32_t first_col, int32_t n_cols, double* s);
 
 /* Eq. 6: patch part of s (after the first n_special entries) as a grid_h x grid_w
  * map, smoothed with a 3x3 Gaussian (sigma = 1, replicate border); aux tokens copied. */

@@ -28,6 +28,7 @@ SCORE_HYBRID = 0
 SCORE_RESIDUAL_STORED = 1
 SCORE_RANDOM = 2
 SCORE_QK = 3
+SCORE_ATTN = 4
 
 
 @dataclasses.dataclass(frozen=True)

@@ -541,6 +541,64 @@ def test_qk_mode_replaces_only_the_current_frame_criterion():
         np.testing.assert_allclose(qk.export(with_kv=False)["stored"][n:], sm, rtol=1e-6)
 
 
+def test_attention_received_is_the_column_mean_of_the_librarys_softmax():
+    """The attention-weight criterion (Supp. D) against torch's softmax of the library matmul's logits: the mean over
+    heads and queries of each key's column.  M, N, H, d all differ.  Over all columns the means add up to 1 (every row
+    of P does); with all-zero queries every key receives exactly 1 / N."""
+    rng = np.random.default_rng(21)
+    M, N, H, d = 5, 17, 3, 8
+    Q = rng.standard_normal((M, H * d)).astype(np.float32)
+    K = rng.standard_normal((N, H * d)).astype(np.float32) * 1.5
+    q = torch.from_numpy(Q).double().view(M, H, d).transpose(0, 1)
+    k = torch.from_numpy(K).double().view(N, H, d).transpose(0, 1)
+    P = torch.softmax(torch.matmul(q, k.transpose(1, 2)) / math.sqrt(d), dim=-1)      # [H, M, N]
+    want = P.mean(dim=(0, 1)).numpy()
+    got = orc.attention_received(Q, K, H)
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-15)
+    assert abs(got.sum() - 1.0) < 1e-12
+    np.testing.assert_allclose(orc.attention_received(Q, K, H, first_col=N - 4, n_cols=4), want[N - 4:], rtol=1e-12)
+    np.testing.assert_allclose(orc.attention_received(np.zeros_like(Q), K, H), np.full(N, 1.0 / N), rtol=1e-14)
+    # a key every query points at collects (nearly) all the attention
+    K2 = K.copy(); K2[3] = 0.0
+    Q2 = np.tile(np.ones((1, H * d), dtype=np.float32) * 3.0, (M, 1)); K2[3] = 3.0
+    assert orc.attention_received(Q2, K2, H)[3] > 0.99
+
+
+def test_attention_weight_mode_scores_the_frame_by_the_attention_it_receives():
+    """The stream in attention-weight mode: the new rows' priorities are beta x min-max of the smoothed attention the
+    frame's tokens receive in the frame's own attention over [cache + frame] (recomputed here with numpy), the cached
+    rows' priorities equal the hybrid mode's, the residual plays no part."""
+    base = gen.config_tiny().replace(anchor_tokens=0, n_frames=6, budget=10_000)
+    cfg = base.replace(score_mode=gen.SCORE_ATTN)
+    aw, hy = orc.OracleLayer.from_stream(cfg), orc.OracleLayer.from_stream(base)
+    M, H, d = cfg.tokens_per_frame, cfg.n_heads, cfg.head_dim
+    for t in range(cfg.n_frames):
+        fi = gen.frame_inputs(cfg, t)
+        aw.attend(t, fi.q, fi.k, fi.v, compute=False)
+        hy.attend(t, fi.q, fi.k, fi.v, compute=False)
+        keys = aw.export()["k"].astype(np.float64)                                     # cache + frame, N rows
+        out = aw.compress(None, fi.conf, fi.rho)
+        ref = hy.compress(fi.resid, fi.conf, fi.rho)
+        n = len(out["r"]) - M
+        if t == 0:
+            continue
+        np.testing.assert_array_equal(out["r"][:n], ref["r"][:n])
+        qh = fi.q.astype(np.float64).reshape(M, H, d).transpose(1, 0, 2)
+        kh = keys.reshape(-1, H, d).transpose(1, 0, 2)
+        logits = qh @ kh.transpose(0, 2, 1) / math.sqrt(d)
+        P = np.exp(logits - logits.max(axis=-1, keepdims=True))
+        P /= P.sum(axis=-1, keepdims=True)
+        s = P.mean(axis=(0, 1))[n:]
+        grid = s[cfg.n_special:].reshape(cfg.grid_h, cfg.grid_w)
+        g = np.exp(-0.5 * np.array([[2, 1, 2], [1, 0, 1], [2, 1, 2]], dtype=np.float64))
+        sm = s.copy()
+        sm[cfg.n_special:] = ((1 - cfg.alpha) * grid + cfg.alpha * scipy.ndimage.correlate(
+            grid, g / g.sum(), mode="nearest")).ravel()
+        want = cfg.beta * (sm - sm.min()) / (sm.max() - sm.min())
+        np.testing.assert_allclose(out["r"][n:], want, rtol=0, atol=2e-6)
+        assert np.abs(out["r"][n:] - ref["r"][n:]).max() > 0.05
+
+
 # ------------------------------------------------------------------ Supp. C: the camera head's cache
 
 def _camera_token(cfg, t, tag):
