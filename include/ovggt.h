@@ -70,8 +70,17 @@ enum { OVGGT_DTYPE_F32 = 0, OVGGT_DTYPE_BF16 = 1 };
  * receives, s_j = 1 / (M n_heads) sum_h sum_i (q_{i,h} . k_{j,h}) / sqrt(head_dim), computed through the column sums
  * of Q.  The attend half computes it from io->q and io->k and keeps it per layer until the layer's compress half,
  * whose io->resid is then not read (it may be NULL); Eq. 6-8 and the key diversity of cached rows are unchanged.
- * Not available for a camera-head cache. */
-enum { OVGGT_SCORE_HYBRID = 0, OVGGT_SCORE_RESIDUAL_STORED = 1, OVGGT_SCORE_RANDOM = 2, OVGGT_SCORE_QK = 3 };
+ * ATTN is the probe's attention-weight baseline, the criterion that needs the attention matrix (reading: the
+ * attention new token j receives in the frame's own attention over [cache + frame], averaged over the frame's M
+ * queries and the heads, s_j = 1 / (M n_heads) sum_h sum_i P_h[i, n + j]).  The attention kernels leave each row's
+ * log2 softmax denominator behind and a second pass over the frame's own M x M block recomputes those columns of P;
+ * it runs in the attend half after the attention, so ovggt_layer_step does not overlap anything in this mode.  The
+ * residual is not read either.
+ * QK and ATTN are not available for a camera-head cache. */
+enum {
+  OVGGT_SCORE_HYBRID = 0, OVGGT_SCORE_RESIDUAL_STORED = 1, OVGGT_SCORE_RANDOM = 2, OVGGT_SCORE_QK = 3,
+  OVGGT_SCORE_ATTN = 4
+};
 enum { OVGGT_FLAG_EVICTABLE = 0, OVGGT_FLAG_INIT = 1, OVGGT_FLAG_HIST = 2 };
 /* Where surviving K/V rows live after Eq. 8 (the paper fixes the survivor set, not a layout):
  *  FILL_HOLES     one K/V buffer per layer; the rows admitted from the new frame are copied into the slots the
@@ -109,7 +118,7 @@ typedef struct {
   const void* k;                /* [M, C] keys of the frame                        (attend) */
   const void* v;                /* [M, C] values of the frame                      (attend) */
   const void* resid;            /* [M, C] FFN residual rows, LayerScale included   (compress, Eq. 5; unused and
-                                   optional in OVGGT_SCORE_QK) */
+                                   optional in OVGGT_SCORE_QK and OVGGT_SCORE_ATTN) */
   const float* conf;            /* [grid_h*grid_w] per-patch confidence, or NULL = no anchor candidate (compress) */
   float rho;                    /* coverage ratio of the latest anchor in this view; NaN = no decision (compress) */
   const float* score_override;  /* [n + M] fp32 or NULL: priorities the selection ranks instead of its own (compress) */

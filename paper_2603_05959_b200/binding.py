@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libovggt_checked.so" if os.environ.get("OVGGT_LI
 MAX_ANCHORS = 16
 
 DTYPE_F32, DTYPE_BF16 = 0, 1
-SCORE_HYBRID, SCORE_RESIDUAL_STORED, SCORE_RANDOM, SCORE_QK = 0, 1, 2, 3
+SCORE_HYBRID, SCORE_RESIDUAL_STORED, SCORE_RANDOM, SCORE_QK, SCORE_ATTN = 0, 1, 2, 3, 4
 FLAG_EVICTABLE, FLAG_INIT, FLAG_HIST = 0, 1, 2
 COMPACT_FILL_HOLES, COMPACT_STABLE_GATHER = 0, 1
 PROF_CLASSES = ["append", "attention", "row_norms", "diversity", "select", "compact"]

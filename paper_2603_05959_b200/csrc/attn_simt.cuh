@@ -14,7 +14,7 @@ constexpr int kSimtTile = 32;    // keys per shared-memory tile
 template <int DT>
 __global__ void __launch_bounds__(kSimtRows) k_attn_simt(const void* __restrict__ q, const void* __restrict__ k,
                                                          const void* __restrict__ v, int M, int N, int H,
-                                                         void* __restrict__ out) {
+                                                         void* __restrict__ out, float* __restrict__ lse = nullptr) {
   constexpr int D = 64, VEC = VecOf<DT>::n, VPR = D / VEC;   // vectors per head-row
   __shared__ __align__(16) float Ks[kSimtTile][D];
   __shared__ __align__(16) float Vs[kSimtTile][D];
@@ -79,6 +79,7 @@ __global__ void __launch_bounds__(kSimtRows) k_attn_simt(const void* __restrict_
   }
   if (m < M) {
     const float inv = 1.0f / l;
+    if (lse != nullptr) lse[(size_t)m * H + h] = mref + log2f(l);   // log2 of the row's softmax denominator
     if constexpr (DT == kBF16) {
       __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out) + (size_t)m * C + (size_t)h * D;
 #pragma unroll

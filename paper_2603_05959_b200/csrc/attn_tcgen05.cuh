@@ -282,6 +282,7 @@ struct AttnParams {
   __nv_bfloat16* out;     // [M, C]            (splits == 1)
   float* o_part;          // [splits, M, C]    un-normalised partial outputs
   float2* ml_part;        // [splits, M, H]    (reference maximum in log2 units, row sum)
+  float* lse;             // [M, H] or nullptr: log2 of each row's softmax denominator (reference + log2 of the sum)
   int* status;
 };
 
@@ -631,6 +632,7 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
       }
       if (P.splits > 1 && m < P.M) P.ml_part[((size_t)split * P.M + m) * P.H + h] = make_float2(mref, l);
+      if (P.splits == 1 && P.lse != nullptr && m < P.M) P.lse[(size_t)m * P.H + h] = mref + log2f(l);
     }
   }
 
@@ -646,7 +648,8 @@ k_attn_tcgen05(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 // out[m, h*64 + c] = sum_s O_s 2^(m_s - m*) / sum_s l_s 2^(m_s - m*), m* = max_s m_s, splits folded in order.
 // One thread per 4 columns; all loads of a thread are issued before the arithmetic that needs them.
 __global__ void __launch_bounds__(256) k_attn_merge(const float* __restrict__ o_part, const float2* __restrict__ ml_part,
-                                                    int M, int H, int splits, __nv_bfloat16* __restrict__ out) {
+                                                    int M, int H, int splits, __nv_bfloat16* __restrict__ out,
+                                                    float* __restrict__ lse) {
   const int C = H * kHD;
   const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   const size_t total = (size_t)M * (C / 4);
@@ -680,6 +683,7 @@ __global__ void __launch_bounds__(256) k_attn_merge(const float* __restrict__ o_
       den = fmaf(w, ml[s].y, den);
     }
   const float inv = 1.0f / den;
+  if (lse != nullptr && (c4 * 4) % kHD == 0) lse[(size_t)m * H + h] = mstar + log2f(den);
   uint2 w;
   w.x = pack_bf16(acc.x * inv, acc.y * inv);
   w.y = pack_bf16(acc.z * inv, acc.w * inv);
@@ -793,7 +797,7 @@ inline int attn_kv_maps(AttnKvMaps* m, const void* k, const void* v, int N, int 
 
 inline int attn_tcgen05_launch(const void* q, const void* k, const void* v, int M, int N, int H, void* out,
                                void* scratch, int* status, cudaStream_t st, AttnKvMaps* kv_maps = nullptr,
-                               int force_splits = 0, const float* kmax2 = nullptr) {
+                               int force_splits = 0, const float* kmax2 = nullptr, float* lse = nullptr) {
   const int C = H * kHD;
   CUtensorMap tq;
   AttnKvMaps local;
@@ -815,6 +819,7 @@ inline int attn_tcgen05_launch(const void* q, const void* k, const void* v, int 
   P.ml_part = reinterpret_cast<float2*>(static_cast<char*>(scratch) + (size_t)kMaxSplits * M * C * 4);
   P.status = status;
   P.kmax2 = kmax2;
+  P.lse = lse;
   cudaError_t e = cudaFuncSetAttribute(k_attn_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemBytes);
   if (e != cudaSuccess) { g_attn_last_error = (int)e; return OVGGT_ERR_CUDA; }
   dim3 grid((M + kBM - 1) / kBM, H, P.splits);
@@ -833,7 +838,8 @@ inline int attn_tcgen05_launch(const void* q, const void* k, const void* v, int 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, k_attn_merge, (const float*)P.o_part, (const float2*)P.ml_part, M, H, P.splits, P.out);
+    e = cudaLaunchKernelEx(&cfg, k_attn_merge, (const float*)P.o_part, (const float2*)P.ml_part, M, H, P.splits, P.out,
+                           lse);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { g_attn_last_error = (int)e; return OVGGT_ERR_CUDA; }
   }

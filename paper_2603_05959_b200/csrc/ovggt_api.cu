@@ -201,6 +201,20 @@ int launch_colsum(const void* K, int rows, int C, int dtype, float* part, float*
   return OVGGT_OK;
 }
 
+// Supp. D, attention-weight criterion: s[j] = mean over the M queries and the heads of the attention key j of the
+// frame received, from the log2 denominators the attention left in lse [M, H] (part: [H, M] floats of scratch).
+int launch_attention_received(const void* q, const void* k, int M, int C, int n_heads, int dtype, const float* lse,
+                              float* part, float* s, cudaStream_t st) {
+  (void)C;
+  dim3 grid((M + kRecvTile - 1) / kRecvTile, n_heads);
+  if (dtype == kBF16) k_attn_received<kBF16><<<grid, 256, 0, st>>>((const uint4*)q, (const uint4*)k, M, n_heads, lse, part);
+  else                k_attn_received<kF32><<<grid, 256, 0, st>>>((const uint4*)q, (const uint4*)k, M, n_heads, lse, part);
+  LAUNCHED();
+  k_fold_heads<<<(M + 255) / 256, 256, 0, st>>>(part, M, n_heads, 1.0f / ((float)M * (float)n_heads), s);
+  LAUNCHED();
+  return OVGGT_OK;
+}
+
 // Supp. D, query-key criterion: s[j] = mean over the M queries and the heads of q_i . k_j / sqrt(d), taken through
 // the column sums of Q (qsum [C] after part [colsum_parts(M), C]; three small kernels).
 int launch_qk_scores(const void* q, const void* k, int M, int C, int n_heads, int dtype, float* part, float* qsum,
@@ -247,15 +261,15 @@ int launch_fill_holes(void* kc, void* vc, const int* msrc, const int* mdst, cons
 
 int launch_attention(const void* q, const void* k, const void* v, int M, int N, int H, int dtype, void* out,
                      void* scratch, int* status, cudaStream_t st, AttnKvMaps* maps = nullptr,
-                     const float* kmax2 = nullptr) {
+                     const float* kmax2 = nullptr, float* lse = nullptr) {
   if (dtype == kBF16) {
-    int rc = attn_tcgen05_launch(q, k, v, M, N, H, out, scratch, status, st, maps, 0, kmax2);
+    int rc = attn_tcgen05_launch(q, k, v, M, N, H, out, scratch, status, st, maps, 0, kmax2, lse);
     if (rc == OVGGT_OK) g_launches.fetch_add(attn_tcgen05_num_launches(M, N, H));
     if (rc == OVGGT_ERR_CUDA) g_last_cuda_error.store(attn_tcgen05_last_error());
     return rc;
   }
   dim3 grid((M + kSimtRows - 1) / kSimtRows, H);
-  k_attn_simt<kF32><<<grid, kSimtRows, 0, st>>>(q, k, v, M, N, H, out);
+  k_attn_simt<kF32><<<grid, kSimtRows, 0, st>>>(q, k, v, M, N, H, out, lse);
   LAUNCHED();
   return OVGGT_OK;
 }
@@ -317,6 +331,7 @@ struct ovggt_cache {
   // shared scratch
   float *colsum_part = nullptr, *ksum = nullptr;
   float *qk_part = nullptr, *qk_sum = nullptr;       // OVGGT_SCORE_QK: column sums of the frame's queries
+  float *attn_lse = nullptr, *attn_part = nullptr;   // OVGGT_SCORE_ATTN: log2 softmax denominators [M, H], per-head sums [H, M]
   void* attn_scratch = nullptr;
   int* status = nullptr;
   // two sets of staging buffers for ovggt_layer_step_host: the copies of one step overlap the kernels of the step before
@@ -394,9 +409,10 @@ bool config_ok(const ovggt_config* c, int* err) {
   if (c->k_max < 0 || c->k_max > OVGGT_MAX_ANCHORS || c->min_anchor_interval < 0) return false;
   if (c->dtype != kF32 && c->dtype != kBF16) return false;
   if (c->score_mode != OVGGT_SCORE_HYBRID && c->score_mode != OVGGT_SCORE_RESIDUAL_STORED &&
-      c->score_mode != OVGGT_SCORE_RANDOM && c->score_mode != OVGGT_SCORE_QK)
+      c->score_mode != OVGGT_SCORE_RANDOM && c->score_mode != OVGGT_SCORE_QK && c->score_mode != OVGGT_SCORE_ATTN)
     return false;
-  if (c->score_mode == OVGGT_SCORE_QK && c->camera_head) return false;   // the probe concerns the aggregator's caches
+  if ((c->score_mode == OVGGT_SCORE_QK || c->score_mode == OVGGT_SCORE_ATTN) && c->camera_head)
+    return false;   // the probe concerns the aggregator's caches
   if (c->compaction != OVGGT_COMPACT_FILL_HOLES && c->compaction != OVGGT_COMPACT_STABLE_GATHER) return false;
   if (!(c->alpha >= 0.0f && c->alpha <= 1.0f) || !(c->beta >= 0.0f && c->beta <= 1.0f)) return false;
   const int64_t M = c->n_special + (int64_t)c->grid_h * c->grid_w;
@@ -488,6 +504,8 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
   const size_t o_status = L.take(64);
   const bool qk = c->score_mode == OVGGT_SCORE_QK;
   const size_t o_qk = qk ? L.take((size_t)(colsum_parts(M) + 1) * C * 4) : 0;
+  const bool aw = c->score_mode == OVGGT_SCORE_ATTN;
+  const size_t o_aw = aw ? L.take((size_t)2 * M * c->n_heads * 4) : 0;
   size_t o_stage[2][5], o_conf[2];
   for (int p = 0; p < 2; ++p) {
     for (int i = 0; i < 5; ++i) o_stage[p][i] = L.take((size_t)M * C * eb);
@@ -498,6 +516,10 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
     h->ksum = reinterpret_cast<float*>(base + o_ksum);
     h->attn_scratch = base + o_attn;
     h->status = reinterpret_cast<int*>(base + o_status);
+    if (aw) {
+      h->attn_lse = reinterpret_cast<float*>(base + o_aw);
+      h->attn_part = h->attn_lse + (size_t)M * c->n_heads;
+    }
     if (qk) {
       h->qk_part = reinterpret_cast<float*>(base + o_qk);
       h->qk_sum = h->qk_part + (size_t)colsum_parts(M) * C;
@@ -517,7 +539,12 @@ size_t layout_workspace(const ovggt_config* c, ovggt_cache* h) {
 
 // Score modes whose cached rows are ranked by key diversity (Eq. 7); the query-key probe (Supp. D) differs from the
 // hybrid mode only in the criterion of the new frame's rows.
-bool ranks_by_diversity(int mode) { return mode == OVGGT_SCORE_HYBRID || mode == OVGGT_SCORE_QK; }
+bool ranks_by_diversity(int mode) {
+  return mode == OVGGT_SCORE_HYBRID || mode == OVGGT_SCORE_QK || mode == OVGGT_SCORE_ATTN;
+}
+// Modes whose criterion for the new frame comes out of the attend half (from q and k, or from the attention itself)
+// and waits in the layer's s_raw; the compress half then does not read the residual.
+bool scored_at_attend(int mode) { return mode == OVGGT_SCORE_QK || mode == OVGGT_SCORE_ATTN; }
 
 int check_layer(ovggt_cache* h, int32_t layer) {
   if (!h) return OVGGT_ERR_INVALID_ARG;
@@ -721,7 +748,8 @@ int enqueue_attention(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, c
   {
     ProfScope ps(h, OVGGT_PROF_ATTENTION, st);
     rc = launch_attention(io->q, S.kbuf[kb], S.vbuf[kb], h->M, S.n + h->M, h->cfg.n_heads, h->cfg.dtype, io->out,
-                          h->attn_scratch, h->status, st, &S.maps[kb], key_norm_bound(h, S));
+                          h->attn_scratch, h->status, st, &S.maps[kb], key_norm_bound(h, S),
+                          h->cfg.score_mode == OVGGT_SCORE_ATTN ? h->attn_lse : nullptr);
   }
   if (rc) return rc;
   if (h->first_frame < 0) {
@@ -741,6 +769,15 @@ int enqueue_qk_scores(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io, c
   return launch_qk_scores(io->q, io->k, h->M, h->C, h->cfg.n_heads, h->cfg.dtype, h->qk_part, h->qk_sum, S.s_raw, st);
 }
 
+// Attention-weight mode (Supp. D): the criterion of the new frame's rows, from the attention that has just been
+// enqueued on st (its log2 denominators) and the frame's own q and k; kept in the layer's s_raw as well.
+int enqueue_received_scores(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io, cudaStream_t st) {
+  if (h->cfg.score_mode != OVGGT_SCORE_ATTN) return OVGGT_OK;
+  ProfScope ps(h, OVGGT_PROF_ROW_NORMS, st);
+  return launch_attention_received(io->q, io->k, h->M, h->C, h->cfg.n_heads, h->cfg.dtype, h->attn_lse, h->attn_part,
+                                   S.s_raw, st);
+}
+
 // Eq. 5 and the diversity score of Sec. 3.2 for the frame io describes: everything the selection needs that does not
 // depend on the anchor decision.  Reads the cached keys [0, n) and the frame's residual, so it may run before the
 // frame's K/V are appended.
@@ -748,8 +785,8 @@ int enqueue_scores(ovggt_cache* h, LayerState& S, const ovggt_frame_io* io, cuda
   const ovggt_config& c = h->cfg;
   const int M = h->M, C = h->C, n = S.n, kb = S.kv;
   const bool hybrid = ranks_by_diversity(c.score_mode) && n > 0;
-  // query-key mode: s_raw was written by the attend half (enqueue_qk_scores); the residual is not read
-  const void* resid = c.score_mode == OVGGT_SCORE_QK ? nullptr : io->resid;
+  // query-key and attention-weight modes: s_raw was written by the attend half; the residual is not read
+  const void* resid = scored_at_attend(c.score_mode) ? nullptr : io->resid;
   int rc = OVGGT_OK;
   if (!hybrid) {
     if (!resid) return OVGGT_OK;
@@ -796,7 +833,7 @@ int validate_compress(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, c
   if (rc) return rc;
   if (!io) return OVGGT_ERR_INVALID_ARG;
   if ((h->cfg.camera_head != 0) != (mirrored != nullptr)) return OVGGT_ERR_INVALID_ARG;
-  if (h->cfg.score_mode != OVGGT_SCORE_QK) {   // (query-key mode does not read the residual)
+  if (!scored_at_attend(h->cfg.score_mode)) {   // (those modes do not read the residual)
     if (!io->resid) return OVGGT_ERR_INVALID_ARG;
     if (!aligned16(io->resid)) return OVGGT_ERR_MISALIGNED;
   }
@@ -855,7 +892,7 @@ CompressParams select_params(ovggt_cache* h, LayerState& S, const ovggt_frame_io
   P.n_special = c.n_special; P.grid_h = c.grid_h; P.grid_w = c.grid_w;
   P.alpha = c.alpha; P.w_center = h->w_center; P.w_edge = h->w_edge; P.w_corner = h->w_corner;
   P.beta = c.beta;
-  P.mode = c.score_mode == OVGGT_SCORE_QK ? OVGGT_SCORE_HYBRID : c.score_mode;   // same Eq. 6-8, other s_raw
+  P.mode = scored_at_attend(c.score_mode) ? OVGGT_SCORE_HYBRID : c.score_mode;   // same Eq. 6-8, other s_raw
   P.protect_new = (first && c.protect_first_frame) ? OVGGT_FLAG_INIT
                                                    : ((c.camera_head && h->decided_register) ? OVGGT_FLAG_HIST : 0);
   P.lone_new = c.camera_head ? 1.0f : -1.0f;
@@ -1005,7 +1042,7 @@ int compress_all_layers(ovggt_cache* h, const ovggt_frame_io* ios, cudaStream_t 
         const bool hybrid = ranks_by_diversity(c.score_mode) && S.n > 0;
         DiversityArgs& A = db.a[i];
         A = DiversityArgs{};
-        A.resid = c.score_mode == OVGGT_SCORE_QK ? nullptr : (const uint4*)ios[l0 + i].resid;
+        A.resid = scored_at_attend(c.score_mode) ? nullptr : (const uint4*)ios[l0 + i].resid;
         A.resid_rows = M; A.s_raw = S.s_raw;
         if (hybrid) {
           const bool fresh = !S.ksum_valid || S.since_refresh >= kColsumRefreshEvery;
@@ -1067,7 +1104,9 @@ extern "C" int ovggt_layer_attend(ovggt_cache* h, int32_t layer, const ovggt_fra
   if (rc) return rc;
   rc = enqueue_attention(h, layer, io, st);
   if (rc) return rc;
-  return enqueue_qk_scores(h, h->layers[layer], io, st);
+  rc = enqueue_qk_scores(h, h->layers[layer], io, st);
+  if (rc) return rc;
+  return enqueue_received_scores(h, h->layers[layer], io, st);
 }
 
 extern "C" int ovggt_layer_compress(ovggt_cache* h, int32_t layer, const ovggt_frame_io* io, void* stream) {
@@ -1102,9 +1141,10 @@ extern "C" int ovggt_layer_step(ovggt_cache* h, int32_t layer, const ovggt_frame
   if (rc) return rc;
   if (h->cfg.camera_head) return OVGGT_ERR_INVALID_ARG;   // the camera head's cache needs the aggregator's decision
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const bool resid_ok = io && (h->cfg.score_mode == OVGGT_SCORE_QK || (io->resid && aligned16(io->resid)));
+  const bool resid_ok = io && (scored_at_attend(h->cfg.score_mode) || (io->resid && aligned16(io->resid)));
+  // (the attention-weight criterion needs the attention's own denominators: nothing to overlap it with)
   const bool can_overlap = h->side && h->overlap && resid_ok && io->q && io->k && io->v && io->out &&
-                           !h->layers[layer].pending;
+                           !h->layers[layer].pending && h->cfg.score_mode != OVGGT_SCORE_ATTN;
   if (!can_overlap) {
     rc = ovggt_layer_attend(h, layer, io, stream);
     if (rc) return rc;

@@ -306,4 +306,89 @@ __global__ void __launch_bounds__(256) k_diversity_batched(const __grid_constant
   diversity_body<DT>(batch.a[blockIdx.y], nvec, sh_ksum);
 }
 
+// Supp. D, attention-weight criterion: part[h, j] = sum_i 2^(c q_i,h . k_j,h - lse[i, h]), the attention key j of the
+// frame receives from the frame's M queries in head h, given each row's log2 softmax denominator over ALL keys (lse,
+// written by the attention kernels).  One CTA per (64 keys, head): the key tile and one 64-query tile at a time sit
+// in shared memory as fp32, thread (ty, tx) of 16 x 16 owns a 4 x 4 block of the 64 x 64 logits.  The sums over i
+// run in a fixed order (query tiles in order, then the 16 thread rows in order), so results are reproducible.
+constexpr int kRecvTile = 64;
+template <int DT>
+__global__ void __launch_bounds__(256) k_attn_received(const uint4* __restrict__ q, const uint4* __restrict__ k, int M,
+                                                       int H, const float* __restrict__ lse, float* __restrict__ part) {
+  constexpr int D = 64, VEC = VecOf<DT>::n, VPR = D / VEC;
+  __shared__ float Ks[kRecvTile][D + 1];
+  __shared__ float Qs[kRecvTile][D + 1];
+  __shared__ float Ls[kRecvTile];
+  __shared__ float red[16][kRecvTile];
+  const int h = blockIdx.y, j0 = blockIdx.x * kRecvTile;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const size_t row_vecs = (size_t)H * VPR;
+  const float c = 1.4426950408889634f * 0.125f;              // log2(e) / sqrt(64)
+  for (int idx = threadIdx.x; idx < kRecvTile * VPR; idx += 256) {
+    const int r = idx / VPR, i = idx - r * VPR;
+    float f[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) f[e] = 0.0f;
+    if (j0 + r < M) unpack<DT>(k[(size_t)(j0 + r) * row_vecs + (size_t)h * VPR + i], f);
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) Ks[r][i * VEC + e] = f[e];
+  }
+  float col[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+  for (int i0 = 0; i0 < M; i0 += kRecvTile) {
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < kRecvTile * VPR; idx += 256) {
+      const int r = idx / VPR, i = idx - r * VPR;
+      float f[VEC];
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) f[e] = 0.0f;
+      if (i0 + r < M) unpack<DT>(q[(size_t)(i0 + r) * row_vecs + (size_t)h * VPR + i], f);
+#pragma unroll
+      for (int e = 0; e < VEC; ++e) Qs[r][i * VEC + e] = f[e];
+    }
+    if (threadIdx.x < kRecvTile) Ls[threadIdx.x] = i0 + threadIdx.x < M ? lse[(size_t)(i0 + threadIdx.x) * H + h] : INFINITY;
+    __syncthreads();
+    float acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) acc[a][b] = 0.0f;
+    for (int d = 0; d < D; ++d) {
+      float qa[4], kb[4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a) qa[a] = Qs[ty * 4 + a][d];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) kb[b] = Ks[tx * 4 + b][d];
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(qa[a], kb[b], acc[a][b]);
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+      const float l2 = Ls[ty * 4 + a];                         // +inf for rows past M: their weight is 2^-inf = 0
+#pragma unroll
+      for (int b = 0; b < 4; ++b) col[b] += exp2f(fmaf(acc[a][b], c, -l2));
+    }
+  }
+#pragma unroll
+  for (int b = 0; b < 4; ++b) red[ty][tx * 4 + b] = col[b];
+  __syncthreads();
+  if (threadIdx.x < kRecvTile && j0 + threadIdx.x < M) {
+    float t = 0.0f;
+#pragma unroll
+    for (int r = 0; r < 16; ++r) t += red[r][threadIdx.x];
+    part[(size_t)h * M + j0 + threadIdx.x] = t;
+  }
+}
+
+// s[j] = scale * sum_h part[h, j], heads in order.
+__global__ void __launch_bounds__(256) k_fold_heads(const float* __restrict__ part, int M, int H, float scale,
+                                                    float* __restrict__ s) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= M) return;
+  float t = 0.0f;
+  for (int h = 0; h < H; ++h) t += part[(size_t)h * M + j];
+  s[j] = t * scale;
+}
+
 }  // namespace ovggt

@@ -68,7 +68,7 @@ def test_workspace_bytes_is_a_pure_host_function(lib):
 def test_create_reports_config_errors_without_a_gpu(lib):
     h = C.c_void_p()
     bad = [(_cfg(head_dim=32), -1), (_cfg(n_layers=0, budget=256), -1), (_cfg(dtype=7), -1),
-           (_cfg(alpha=1.5), -1), (_cfg(k_max=17), -1), (_cfg(anchor_tokens=65), -1), (_cfg(compaction=2), -1), (_cfg(score_mode=4), -1),
+           (_cfg(alpha=1.5), -1), (_cfg(k_max=17), -1), (_cfg(anchor_tokens=65), -1), (_cfg(compaction=2), -1), (_cfg(score_mode=5), -1),
            (_cfg(camera_head=1, n_special=1, grid_h=0, grid_w=0, anchor_tokens=0, budget=8, score_mode=3), -1),
            (_cfg(camera_head=1), -1), (_cfg(camera_head=1, n_special=1, grid_h=0, grid_w=0, anchor_tokens=0, budget=3), -3),
            (_cfg(budget=68), -3), (_cfg(budget=69 + 3 * 8 - 1), -3)]
