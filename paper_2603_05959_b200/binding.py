@@ -66,6 +66,9 @@ class OvggtStats(C.Structure):
     ]
 
 
+ERR_TIMEOUT, ERR_UNSUPPORTED, ERR_TOO_LARGE = -9, -10, -11      # (the codes of include/ovggt.h that callers test for)
+
+
 class OvggtError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code

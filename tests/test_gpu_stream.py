@@ -177,6 +177,33 @@ def test_query_key_mode_through_the_overlapped_step_and_the_batched_compress():
         cache.destroy()
 
 
+def test_largest_budget_the_selection_cluster_holds():
+    """Maximum size.  The fused selection kernel keeps all B + M candidates of a layer in the shared memory of one
+    8-CTA cluster; ovggt_cache_create refuses a budget beyond that with OVGGT_ERR_UNSUPPORTED.  The largest budget it
+    accepts for 2000-token frames (found by asking) is filled and then evicts for five frames, teacher-forced:
+    survivors and layout bit-exact, the library's own priorities within tolerance, at about 75,000 candidates."""
+    base = gen.StreamConfig(name="max", n_heads=1, n_special=20, grid_h=45, grid_w=44, anchor_tokens=16,
+                            min_anchor_interval=5, tau=0.6, budget=0)
+
+    def accepted(budget):
+        try:
+            B.OvggtCache.from_stream(base.replace(budget=budget)).destroy()
+            return True
+        except B.OvggtError as e:
+            assert e.code == B.ERR_UNSUPPORTED, e
+            return False
+
+    lo, hi = 40_000, 200_000                    # accepted, refused
+    assert accepted(lo) and not accepted(hi)
+    while hi - lo > 500:
+        mid = (lo + hi) // 2
+        lo, hi = (mid, hi) if accepted(mid) else (lo, mid)
+    assert 60_000 <= lo <= 100_000, lo
+    cfg = base.replace(budget=lo, n_frames=lo // base.tokens_per_frame + 6)
+    layer = run_teacher_forced(cfg, cfg.n_frames, attn_frames=set(), export_every=10_000)
+    assert layer.evicted_total >= 4 * cfg.tokens_per_frame and layer.n_rows == lo
+
+
 @BOTH_LAYOUTS
 def test_attention_weight_mode_matches_the_oracle(compaction):
     """The attention-weight criterion of the scoring probe (Supp. D): the attention the frame's tokens receive in
