@@ -43,7 +43,8 @@ def lib():
         spec = importlib.util.spec_from_file_location("_oracle_build", os.path.join(_HERE, "build.py"))
         mod = importlib.util.module_from_spec(spec)
         spec.loader.exec_module(mod)
-        L = C.CDLL(mod.build())
+        # (OVGGT_ORACLE_LIBRARY: another build of the oracle, for the test that plants mistakes in copies of it)
+        L = C.CDLL(os.environ.get("OVGGT_ORACLE_LIBRARY") or mod.build())
         L.orc_create.restype = C.c_void_p
         L.orc_create.argtypes = [C.POINTER(OrcConfig)]
         L.orc_destroy.argtypes = [C.c_void_p]
